@@ -1,0 +1,166 @@
+/*
+ * worldkv-b200: C ABI of the WorldKV hot path on one B200 (sm_100a).
+ *
+ * The calls follow the paper's statement of the method:
+ *   - World Compression (Section 4.3, Eq. 5): wk_compress_chunk
+ *   - the chunk pool of evicted KV chunks (Section 4.2):  wk_pool_append / wk_pool_evict
+ *   - World Retrieval (Section 4.2 Eq. 4, distance of Section 5.1): wk_retrieve
+ *   - attention of the denoising chunk over [window + retrieved chunks] (Section 4.2): wk_memory_attention
+ *
+ * Conventions
+ *   - All tensor arguments are DEVICE pointers unless the name ends in _host.  bf16 tensors are
+ *     token-major: one row per token holding all heads, [tokens][n_heads][head_dim], row stride
+ *     D = n_heads * head_dim elements, base address 16-byte aligned.
+ *   - Every call returns a wk_status: 0 on success, negative on error.  Errors that can be told from
+ *     the arguments are returned before anything is launched and leave all state untouched.
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = legacy default
+ *     stream) and is asynchronous.  Anomalies only the device can see (a stale slot id, a bounded
+ *     wait that ran out, a non-finite score) set bits in a status word read with wk_poll_status.
+ *   - Ownership: the caller owns every device buffer, including pool storage and scratch (sizes come
+ *     from wk_pool_bytes / wk_scratch_bytes; the context only keeps host-side bookkeeping and tensor
+ *     maps).  No call allocates device memory.  One context may be used by one host thread at a time.
+ *   - There is no CPU fallback: without a CUDA device of compute capability 10.x, wk_create fails.
+ */
+#ifndef WK_H_
+#define WK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t wk_status;
+enum {
+  WK_OK = 0,
+  WK_ERR_ARG = -1,        /* NULL pointer, misaligned pointer, negative count, bad config field */
+  WK_ERR_SHAPE = -2,      /* a size outside what the context was created for */
+  WK_ERR_POOL_FULL = -3,  /* wk_pool_append with no free slot */
+  WK_ERR_BAD_SLOT = -4,   /* host-visible slot id out of range or not valid */
+  WK_ERR_CUDA = -5,       /* a CUDA runtime/driver call failed (wk_last_cuda_error has the code) */
+  WK_ERR_TIMEOUT = -6,    /* reported by wk_poll_status: a bounded device wait ran out */
+  WK_ERR_NONFINITE = -7,  /* reported by wk_poll_status: a score was NaN/Inf */
+  WK_ERR_UNBOUND = -8,    /* wk_bind has not been called */
+  WK_ERR_NO_DEVICE = -9   /* no sm_100-class device */
+};
+
+/* bits of the device status word (wk_poll_status) */
+enum { WK_DEV_BAD_SLOT = 1u, WK_DEV_TIMEOUT = 2u, WK_DEV_NONFINITE = 4u };
+
+typedef struct wk_ctx wk_ctx;
+
+typedef struct {
+  int32_t n_layers;
+  int32_t n_heads;
+  int32_t head_dim;          /* must be 128 */
+  int32_t tokens_per_frame;  /* T */
+  int32_t frames_per_chunk;  /* F (the paper uses 3); frame 0 of a chunk is the anchor */
+  int32_t n_keep;            /* kept non-anchor tokens per chunk, 0 .. (F-1)*T; the paper's P = 25 % is (F-1)*T/4 */
+  int32_t pool_slots;        /* capacity of the chunk pool, in chunks */
+  int32_t max_k;             /* largest retrieval budget / slot list length */
+  int32_t max_dense_segments;/* 1..8 */
+  int32_t device;            /* CUDA device ordinal */
+  float softmax_scale;       /* 0 selects 1/sqrt(head_dim) */
+  int32_t reserved;          /* must be 0 */
+} wk_config;
+
+/* ---- context ------------------------------------------------------------------------------- */
+
+/* Validates the config, selects the device and creates host-side state.  No device memory is taken. */
+wk_status wk_create(const wk_config* cfg, wk_ctx** out);
+void wk_destroy(wk_ctx* ctx);
+
+/* Bytes of pool storage for this config: K and V rows of every slot of every layer
+ * ([n_layers][pool_slots][T + n_keep][D] bf16, twice), slot poses and validity flags. */
+size_t wk_pool_bytes(const wk_config* cfg);
+/* Bytes of scratch: per-problem mean anchor vectors and scores for up to max_batch compression
+ * problems per call, and fp32 split-KV partials for queries of up to max_lq tokens with up to
+ * max_splits KV splits. */
+size_t wk_scratch_bytes(const wk_config* cfg, int32_t max_batch, int32_t max_lq, int32_t max_splits);
+/* Hands the context its two caller-owned device buffers (256-byte aligned).  The pool buffer must be
+ * zero-filled by the caller the first time (all slots invalid).  Clears a few hundred bytes of the
+ * scratch buffer with a synchronous cudaMemset; enqueues nothing else. */
+wk_status wk_bind(wk_ctx* ctx, void* pool_dev, size_t pool_bytes, void* scratch_dev, size_t scratch_bytes,
+                  int32_t max_batch, int32_t max_lq, int32_t max_splits);
+
+/* ---- World Compression (Section 4.3, Eq. 5) ----------------------------------------------- */
+
+/* For each of `batch` independent (layer, chunk) problems: the score of every non-anchor key is its
+ * mean cosine similarity to the T anchor-frame keys (whole-token keys, all heads concatenated); the
+ * n_keep lowest pooled scores are kept, ties to the lowest index.
+ *   K_chunks     [batch] problems, problem b at K_chunks + b * batch_stride_elems, each [F*T][D] bf16
+ *   keep_idx_out [batch][T + n_keep] int32: chunk-local token indices, ascending (anchors 0..T-1 first)
+ *   scores_out   [batch][(F-1)*T] fp32 or NULL: the fp32 first-pass scores, for inspection only;
+ *                the selection itself is decided on fp64 values near the threshold
+ * Errors: WK_ERR_ARG, WK_ERR_SHAPE (batch > max_batch), WK_ERR_UNBOUND. */
+wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_stride_elems, int32_t batch,
+                            int32_t* keep_idx_out, float* scores_out, void* stream);
+
+/* ---- chunk pool (Section 4.2) -------------------------------------------------------------- */
+
+/* Stores one chunk: for layers layer0 .. layer0+n-1 gathers rows keep_idx[l][0 .. T+n_keep) of that
+ * layer's K and V chunk into the lowest free slot, and records the chunk's pose
+ * [tx, ty, tz, 0, qw, qx, qy, qz].  A chunk may be appended in several calls covering different layer
+ * ranges: the first call (slot_io_host = -1 on entry) picks the slot and returns it; later calls pass it
+ * back.  The slot becomes visible to wk_retrieve / wk_memory_attention once every layer is stored.
+ *   K_chunks, V_chunks  layer l at + (l - layer0) * batch_stride_elems, each [F*T][D] bf16
+ *   keep_idx_dev        [n][T + n_keep] int32 (the output of wk_compress_chunk)
+ * Errors: WK_ERR_POOL_FULL, WK_ERR_BAD_SLOT (slot_io_host not an open append), WK_ERR_SHAPE, WK_ERR_ARG. */
+wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
+                         int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,
+                         int64_t chunk_tag, int32_t* slot_io_host, void* stream);
+/* Frees a slot (stream-ordered: kernels already enqueued still see it).  WK_ERR_BAD_SLOT if not valid. */
+wk_status wk_pool_evict(wk_ctx* ctx, int32_t slot, void* stream);
+int32_t wk_pool_oldest(const wk_ctx* ctx);   /* valid slot with the earliest append, -1 if empty */
+int32_t wk_pool_count(const wk_ctx* ctx);    /* number of valid slots */
+int64_t wk_pool_tag(const wk_ctx* ctx, int32_t slot); /* chunk_tag given at append, -1 if not valid */
+
+/* ---- World Retrieval (Section 4.2 Eq. 4; Section 5.1) -------------------------------------- */
+
+/* Distance of every stored chunk's pose to cur_pose: squared-L2 translation distance and geodesic
+ * rotation angle, each divided by its maximum over the stored chunks, summed.  Writes the min(k, M)
+ * slots with the smallest distance, ties to the lowest slot, in rank order.
+ *   slots_out_dev [max_k] int32 (entries past the count are set to -1); dist_out_dev [max_k] fp64 or NULL
+ *   n_out_host    the count min(k, M), known on the host
+ * Errors: WK_ERR_SHAPE (k > max_k or k < 0), WK_ERR_ARG, WK_ERR_UNBOUND. */
+wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_t* slots_out_dev,
+                      double* dist_out_dev, int32_t* n_out_host, void* stream);
+
+/* ---- memory attention (Section 4.2) -------------------------------------------------------- */
+
+typedef struct {
+  const void* K;      /* [n_tokens][H][128] bf16 */
+  const void* V;      /* [n_tokens][H][128] bf16 */
+  int32_t n_tokens;   /* > 0 */
+  int32_t reserved;   /* 0 */
+} wk_dense_seg;
+
+/* O = softmax(scale * Q K^T) V per head, unmasked, over the dense segments (denoising chunk, window,
+ * sink ...) followed by the stored rows of each listed pool slot of `layer`.  Nothing is concatenated
+ * in memory: K/V tiles are fetched where they lie.
+ *   Q [lq][H][128] bf16, O same shape; lse_out [H][lq] fp32 (natural log) or NULL
+ *   slots_dev [n_slots] int32 in device memory (e.g. wk_retrieve's output); an entry that is -1 is
+ *             skipped silently, any other out-of-range or invalid entry is skipped and sets
+ *             WK_DEV_BAD_SLOT; a slot listed twice is attended twice
+ *   kv_splits 0 = choose automatically; otherwise 1 .. max_splits
+ * Errors: WK_ERR_SHAPE (lq > max_lq, n_slots > max_k, n_segs > max_dense_segments, kv_splits > max_splits),
+ * WK_ERR_ARG (no KV at all: n_segs = 0 and n_slots = 0), WK_ERR_UNBOUND, WK_ERR_CUDA. */
+wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, const wk_dense_seg* segs_host,
+                              int32_t n_segs, const int32_t* slots_dev, int32_t n_slots, void* O, float* lse_out,
+                              int32_t kv_splits, void* stream);
+
+/* ---- status -------------------------------------------------------------------------------- */
+
+/* Synchronises the stream, reads and clears the device status word.  Returns WK_OK when no bit is set,
+ * else the error of the most severe bit; *device_flags (may be NULL) receives the raw bits. */
+wk_status wk_poll_status(wk_ctx* ctx, uint32_t* device_flags, void* stream);
+const char* wk_status_string(wk_status s);
+int32_t wk_last_cuda_error(const wk_ctx* ctx);
+/* Number of kernels this context has launched since creation (for benchmark bookkeeping). */
+int64_t wk_launch_count(const wk_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WK_H_ */

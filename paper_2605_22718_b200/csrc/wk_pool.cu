@@ -1,0 +1,63 @@
+// Chunk pool (Section 4.2): device side of append (row-gather compaction of K and V into a slot) and of the
+// slot table (validity flag + pose).  Slot allocation and FIFO bookkeeping are host side (wk_api.cu).
+#include "wk_internal.cuh"
+
+namespace wk {
+namespace {
+
+constexpr int kAppendThreads = 256;
+
+// grid = (ceil(C / rows_per_cta), n_layers_in_call, 2 [K|V]); one warp per kept row, 16-byte vectors.
+__global__ void __launch_bounds__(kAppendThreads)
+append_rows(const __nv_bfloat16* __restrict__ Ksrc, const __nv_bfloat16* __restrict__ Vsrc, int64_t stride,
+            const int32_t* __restrict__ keep_idx, int C, int FT, int D, __nv_bfloat16* __restrict__ Kdst,
+            __nv_bfloat16* __restrict__ Vdst, int64_t dst_layer_stride, int rows_per_cta, uint32_t* __restrict__ status) {
+  const int l = blockIdx.y, which = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const __nv_bfloat16* src = (which ? Vsrc : Ksrc) + static_cast<int64_t>(l) * stride;
+  __nv_bfloat16* dst = (which ? Vdst : Kdst) + static_cast<int64_t>(l) * dst_layer_stride;
+  const int32_t* idx = keep_idx + static_cast<int64_t>(l) * C;
+  const int vecs = D >> 3;
+  const int r0 = blockIdx.x * rows_per_cta, r1 = min(C, r0 + rows_per_cta);
+  for (int r = r0 + warp; r < r1; r += kAppendThreads / 32) {
+    const int j = idx[r];
+    if (j < 0 || j >= FT) {                       // never dereference a bad index
+      if (lane == 0) atomicOr(status, WK_DEV_BAD_SLOT);
+      continue;
+    }
+    const uint4* s = reinterpret_cast<const uint4*>(src + static_cast<int64_t>(j) * D);
+    uint4* d = reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * D);
+    for (int v = lane; v < vecs; v += 32) d[v] = __ldg(s + v);
+  }
+}
+
+struct Pose8 { float v[8]; };
+
+__global__ void slot_mark(int32_t* __restrict__ valid, float* __restrict__ poses, int slot, int is_valid, Pose8 pose) {
+  if (threadIdx.x < 8) poses[slot * 8 + threadIdx.x] = pose.v[threadIdx.x];
+  if (threadIdx.x == 0) valid[slot] = is_valid;
+}
+
+}  // namespace
+
+wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfloat16* K, const __nv_bfloat16* V,
+                        int64_t stride, const int32_t* keep_idx, cudaStream_t s) {
+  const int C = ctx->C, D = ctx->D;
+  const int64_t slot_elems = static_cast<int64_t>(C) * D;
+  const int64_t layer_stride = slot_elems * ctx->cfg.pool_slots;
+  __nv_bfloat16* Kdst = ctx->Kpool + layer0 * layer_stride + slot * slot_elems;
+  __nv_bfloat16* Vdst = ctx->Vpool + layer0 * layer_stride + slot * slot_elems;
+  const int rows_per_cta = 32;
+  const dim3 grid((C + rows_per_cta - 1) / rows_per_cta, n, 2);
+  append_rows<<<grid, kAppendThreads, 0, s>>>(K, V, stride, keep_idx, C, ctx->FT, D, Kdst, Vdst, layer_stride,
+                                              rows_per_cta, ctx->status_dev);
+  return after_launch(ctx);
+}
+
+wk_status launch_slot_mark(wk_ctx* ctx, int slot, int valid, const float* pose, cudaStream_t s) {
+  Pose8 p;
+  for (int i = 0; i < 8; ++i) p.v[i] = pose[i];
+  slot_mark<<<1, 32, 0, s>>>(ctx->valid_dev, ctx->poses_dev, slot, valid, p);
+  return after_launch(ctx);
+}
+
+}  // namespace wk

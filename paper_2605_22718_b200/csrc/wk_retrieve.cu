@@ -1,0 +1,94 @@
+// World Retrieval (Section 4.2, Eq. 4) with the camera distance of Section 5.1: squared-L2 translation
+// distance and geodesic rotation angle to the current pose, each divided by its maximum over the stored
+// chunks, summed; the k smallest win, ties to the lowest slot.  The whole pool is a few KB of poses, so one
+// CTA does everything in fp64 in a single launch and the result stays in device memory for the attention call.
+#include "wk_internal.cuh"
+
+namespace wk {
+namespace {
+
+constexpr int kRetrieveThreads = 1024;
+
+struct Pose8 { float v[8]; };
+
+__device__ __forceinline__ double block_max(double v, double* red) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  double r = red[0];
+  for (int w = 1; w < kRetrieveThreads / 32; ++w) r = fmax(r, red[w]);
+  return r;
+}
+
+__global__ void __launch_bounds__(kRetrieveThreads)
+retrieve_kernel(const float* __restrict__ poses, const int32_t* __restrict__ valid, int n_slots, Pose8 cur, int k,
+                int max_k, double* __restrict__ dist /*[2][n_slots]*/, int32_t* __restrict__ slots_out,
+                double* __restrict__ dist_out) {
+  __shared__ double red[kRetrieveThreads / 32];
+  const int tid = threadIdx.x;
+  double* dt = dist;
+  double* dr = dist + n_slots;
+  double mt = 0.0, mr = 0.0;
+  for (int s = tid; s < n_slots; s += kRetrieveThreads) {
+    if (!valid[s]) { dt[s] = -1.0; continue; }     // negative marks "not a candidate"
+    const float* p = poses + s * 8;
+    const double dx = static_cast<double>(p[0]) - static_cast<double>(cur.v[0]);
+    const double dy = static_cast<double>(p[1]) - static_cast<double>(cur.v[1]);
+    const double dz = static_cast<double>(p[2]) - static_cast<double>(cur.v[2]);
+    const double t = dx * dx + dy * dy + dz * dz;
+    const double dot = static_cast<double>(p[4]) * cur.v[4] + static_cast<double>(p[5]) * cur.v[5] +
+                       static_cast<double>(p[6]) * cur.v[6] + static_cast<double>(p[7]) * cur.v[7];
+    const double r = 2.0 * acos(fmin(1.0, fabs(dot)));    // q and -q are the same rotation
+    dt[s] = t;
+    dr[s] = r;
+    mt = fmax(mt, t);
+    mr = fmax(mr, r);
+  }
+  mt = block_max(mt, red);
+  mr = block_max(mr, red);
+  __syncthreads();
+  // combined distance, each term normalised by its maximum over the candidates (a zero maximum drops the term)
+  for (int s = tid; s < n_slots; s += kRetrieveThreads) {
+    if (dt[s] < 0.0) continue;
+    const double a = mt > 0.0 ? dt[s] / mt : 0.0;
+    const double b = mr > 0.0 ? dr[s] / mr : 0.0;
+    dr[s] = a + b;
+  }
+  for (int i = tid; i < max_k; i += kRetrieveThreads) {
+    slots_out[i] = -1;
+    if (dist_out) dist_out[i] = 0.0;
+  }
+  __syncthreads();
+  // rank by counting: position of slot s = number of candidates that precede it under (distance, slot)
+  for (int s = tid; s < n_slots; s += kRetrieveThreads) {
+    if (dt[s] < 0.0) continue;
+    const double d = dr[s];
+    int rank = 0;
+    for (int u = 0; u < n_slots; ++u) {
+      if (dt[u] < 0.0) continue;
+      const double du = dr[u];
+      rank += (du < d) || (du == d && u < s);
+    }
+    if (rank < k) {
+      slots_out[rank] = s;
+      if (dist_out) dist_out[rank] = d;
+    }
+  }
+}
+
+}  // namespace
+
+wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out,
+                          cudaStream_t s) {
+  Pose8 cur;
+  for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose[i];
+  double* dist = reinterpret_cast<double*>(ctx->scratch_base + ctx->sl.dist_off);
+  retrieve_kernel<<<1, kRetrieveThreads, 0, s>>>(ctx->poses_dev, ctx->valid_dev, ctx->cfg.pool_slots, cur, k,
+                                                 ctx->cfg.max_k, dist, slots_out, dist_out);
+  return after_launch(ctx);
+}
+
+}  // namespace wk
