@@ -1,0 +1,430 @@
+#!/usr/bin/env python
+"""Benchmark of the WorldKV hot path on B200: one "step" = one chunk step of the full denoising pass
+(workload cfg2: 30 layers x 4 denoising steps of memory attention over window + top-8 retrieved chunks from a
+250-chunk compressed pool, plus retrieval, and compression + pool append of the chunk leaving the window).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2|cfg1|cfg3|cfg0]
+
+Prints ONE JSON line.  `value` = attention FLOPs of a chunk step / chunk-step time (whole hot path in the
+denominator), inputs resident in HBM; `e2e` = the same with the step's inputs copied from pinned host memory and
+its outputs copied back inside the timed region.  `--impl reference` times the CPU oracle on a bounded sample.
+With N > 1 (torchrun) every rank runs an independent replica of the workload (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import wkinputs as wi  # noqa: E402
+
+METRIC = "memory-attn TFLOP/s over the whole chunk step (attention + retrieval + compression + pool append)"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per memory_attention_kernel launch from the ncu capture summarised in
+# profiles/ (cfg2 shape, one layer call); None until a capture has been taken for the current kernel.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            res.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return res
+
+
+# ------------------------------------------------------------------------------------------ distributed helpers
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value_ms: float, device) -> float:
+    """Largest of the ranks' timings (every rank gets it)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return value_ms
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+# ------------------------------------------------------------------------------------------ workload on the device
+class ChunkStepBench:
+    """Holds the pool, the per-layer window buffers and rotating inputs of one workload, and runs chunk steps."""
+
+    def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True):
+        import torch
+        from paper_2605_22718_b200 import WorldKV
+        from wkinputs import device as wd
+        self.torch, self.wd, self.w = torch, wd, w
+        self.dev = torch.device("cuda", device_index)
+        torch.cuda.set_device(self.dev)
+        L, H, T, D = w.n_layers, w.n_heads, w.T, w.D
+        self.kv = WorldKV(n_layers=L, n_heads=H, tokens_per_frame=T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
+                          max_k=max(w.k, 1), max_dense_segments=2, device=device_index, max_batch=L, max_lq=w.Lq,
+                          max_splits=8)
+        bf = torch.bfloat16
+        n_poses = w.pool_chunks + 4096
+        if w.trajectory == "actions":
+            self.poses = wi.action_rollout_poses(w.seed, n_poses)
+        elif w.trajectory == "loop":
+            self.poses = wi.loop_poses(w.seed, w.pool_chunks + 3)
+        else:
+            self.poses = wi.random_poses(w.seed, n_poses)
+        # pool pre-fill through the product path: generate -> compress -> append, all layers of a chunk per call
+        Kc = torch.empty((L, w.F * T, D), dtype=bf, device=self.dev)
+        Vc = torch.empty((L, w.F * T, D), dtype=bf, device=self.dev)
+        self.keep = torch.empty((L, w.C), dtype=torch.int32, device=self.dev)
+        for c in range(w.pool_chunks):
+            for l in range(L):
+                wd.key_chunk(Kc[l], w.seed, l, c, T, D, w.sigma, w.F)
+                wd.value_chunk(Vc[l], w.seed, l, c, T, D, w.F)
+            self.kv.compress_chunk(Kc, keep_idx_out=self.keep)
+            self.kv.pool_append(0, L, Kc, Vc, self.keep, self.poses[c % len(self.poses)], chunk_tag=c)
+        # chunks leaving the window: a few distinct input sets, rotated
+        self.evK = [torch.empty((L, w.F * T, D), dtype=bf, device=self.dev) for _ in range(evict_sets)]
+        self.evV = [torch.empty((L, w.F * T, D), dtype=bf, device=self.dev) for _ in range(evict_sets)]
+        for i in range(evict_sets):
+            for l in range(L):
+                wd.key_chunk(self.evK[i][l], w.seed, l, w.pool_chunks + i, T, D, w.sigma, w.F)
+                wd.value_chunk(self.evV[i][l], w.seed, l, w.pool_chunks + i, T, D, w.F)
+        # per-layer dense segments: the denoising chunk and the native window
+        nwin = w.window_frames * T
+        self.curK = torch.empty((L, w.Lq, H, 128), dtype=bf, device=self.dev)
+        self.curV = torch.empty((L, w.Lq, H, 128), dtype=bf, device=self.dev)
+        self.winK = torch.empty((L, max(nwin, 1), H, 128), dtype=bf, device=self.dev)
+        self.winV = torch.empty((L, max(nwin, 1), H, 128), dtype=bf, device=self.dev)
+        base = w.pool_chunks + evict_sets
+        for l in range(L):
+            wd.fill_normal_bf16(self.curV[l], w.seed, wi.STREAM_V + l, (base + 3) * w.F * T * D)
+            tmp = torch.empty((w.F * T, D), dtype=bf, device=self.dev)
+            wd.key_chunk(tmp, w.seed, l, base + 3, T, D, w.sigma, w.F)
+            self.curK[l].view(-1, D)[:] = tmp[:w.Lq]
+            for j in range((nwin + w.F * T - 1) // (w.F * T)):
+                r0, r1 = j * w.F * T, min(nwin, (j + 1) * w.F * T)
+                wd.key_chunk(tmp, w.seed, l, base + 1 + j, T, D, w.sigma, w.F)
+                self.winK[l].view(-1, D)[r0:r1] = tmp[:r1 - r0]
+                wd.value_chunk(tmp, w.seed, l, base + 1 + j, T, D, w.F)
+                self.winV[l].view(-1, D)[r0:r1] = tmp[:r1 - r0]
+        # one Q and one O per (layer, denoising step): rotating buffers far larger than L2
+        S = w.denoise_steps
+        self.Q = torch.empty((L, S, w.Lq, H, 128), dtype=bf, device=self.dev)
+        for l in range(L):
+            for s in range(S):
+                wd.query(self.Q[l, s], w.seed, l, s, 0)
+        self.O = torch.empty_like(self.Q)
+        self.slots = torch.full((max(w.k, 1),), -1, dtype=torch.int32, device=self.dev)
+        self.step_no = 0
+        self.attn_events = []
+        self.e2e = e2e
+        if e2e:
+            self.hQ = torch.empty(self.Q.shape, dtype=bf, pin_memory=True)
+            self.hQ.copy_(self.Q)
+            self.hcurK = torch.empty(self.curK.shape, dtype=bf, pin_memory=True)
+            self.hcurK.copy_(self.curK)
+            self.hcurV = torch.empty(self.curV.shape, dtype=bf, pin_memory=True)
+            self.hcurV.copy_(self.curV)
+            self.hO = torch.empty(self.O.shape, dtype=bf, pin_memory=True)
+        torch.cuda.synchronize(self.dev)
+        st, flags = self.kv.poll_status()
+        if st != 0:
+            raise RuntimeError(f"device status after setup: {st} flags {flags}")
+
+    def attention_flops_per_call(self) -> float:
+        return self.w.attention_flops()
+
+    def attention_calls_per_step(self) -> int:
+        return self.w.n_layers * self.w.denoise_steps
+
+    def step(self, record_attention_events: bool = False, host_io: bool = False):
+        torch, w, kv = self.torch, self.w, self.kv
+        i = self.step_no
+        self.step_no += 1
+        if host_io:   # the step's inputs arrive from pinned host memory
+            self.Q.copy_(self.hQ, non_blocking=True)
+            self.curK.copy_(self.hcurK, non_blocking=True)
+            self.curV.copy_(self.hcurV, non_blocking=True)
+        pose = self.poses[(w.pool_chunks + i) % len(self.poses)]
+        _, n = kv.retrieve(pose, w.k, slots_out=self.slots)
+        if record_attention_events:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+        for s in range(w.denoise_steps):
+            for l in range(w.n_layers):
+                segs = [(self.curK[l], self.curV[l])]
+                if w.window_frames > 0:
+                    segs.append((self.winK[l], self.winV[l]))
+                kv.memory_attention(l, self.Q[l, s], segs, self.slots, n, O=self.O[l, s])
+        if record_attention_events:
+            e1.record()
+            self.attn_events.append((e0, e1))
+        # the chunk leaving the window: compress every layer, evict the oldest stored chunk, append
+        j = i % len(self.evK)
+        kv.compress_chunk(self.evK[j], keep_idx_out=self.keep)
+        if kv.pool_count() == w.pool_chunks:
+            kv.pool_evict(kv.pool_oldest())
+        kv.pool_append(0, w.n_layers, self.evK[j], self.evV[j], self.keep, pose, chunk_tag=w.pool_chunks + i)
+        if host_io:   # and its result goes back
+            self.hO.copy_(self.O, non_blocking=True)
+
+    def time_steps(self, steps: int, host_io: bool):
+        torch = self.torch
+        barrier()
+        torch.cuda.synchronize(self.dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.step(record_attention_events=not host_io, host_io=host_io)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        barrier()
+        return e0.elapsed_time(e1)
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle legs
+class OracleSample:
+    """The oracle, as it stands, on a bounded sample of the workload: some query rows of one attention call over the
+    full KV set of one layer, one compression problem, one retrieval.  Inputs are generated once (untimed)."""
+
+    def __init__(self, w: wi.Workload):
+        from oracle import worldkv_oracle as o
+        self.o, self.w = o, w
+        try:
+            from threadpoolctl import threadpool_info
+            self.threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            self.threads = os.cpu_count() or 1
+        T, D, H = w.T, w.D, w.n_heads
+        self.k = min(w.k, 8)
+        self.pool = o.PoolModel(n_slots=self.k, n_layers=1)
+        self.poses = wi.random_poses(w.seed, self.k + 1)
+        self.K0 = None
+        for c in range(self.k):
+            K = wi.key_chunk_bf16(w.seed, 0, c, T, D, w.sigma, w.F)
+            V = wi.value_chunk_bf16(w.seed, 0, c, T, D, w.F)
+            if self.K0 is None:
+                self.K0 = K
+            idx, _, _ = o.compress_chunk(K, T, w.n_keep)
+            self.pool.append([K.reshape(-1, H, 128)], [V.reshape(-1, H, 128)], [idx], self.poses[c])
+        n_dense = w.Lq + w.window_frames * T
+        reps = (n_dense + w.F * T - 1) // (w.F * T)
+        Kd = np.concatenate([wi.key_chunk_bf16(w.seed, 0, 100 + r, T, D, w.sigma, w.F) for r in range(reps)])[:n_dense]
+        Vd = np.concatenate([wi.value_chunk_bf16(w.seed, 0, 100 + r, T, D, w.F) for r in range(reps)])[:n_dense]
+        self.dense = [(Kd.reshape(-1, H, 128), Vd.reshape(-1, H, 128))]
+        self.Q = wi.query_bf16(w.seed, 0, 0, 0, w.Lq, D).reshape(w.Lq, H, 128)
+        self.many_poses = wi.random_poses(w.seed + 1, w.pool_chunks)
+        self.lkv = n_dense + self.k * w.C
+
+    def run(self, attn_rows: int):
+        o, w = self.o, self.w
+        attn_rows = min(attn_rows, w.Lq)
+        rows = np.linspace(0, w.Lq - 1, attn_rows).astype(np.int64)
+        t0 = time.perf_counter()
+        o.compress_chunk(self.K0, w.T, w.n_keep)
+        t_compress = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        o.retrieve(self.poses[self.k], self.many_poses, list(range(w.pool_chunks)), w.k)
+        t_retrieve = time.perf_counter() - t0
+        t0 = time.perf_counter()
+        o.memory_attention(self.Q, self.dense, self.pool, 0, list(range(self.k)), rows=rows)
+        t_attn = time.perf_counter() - t0
+        calls = w.n_layers * w.denoise_steps
+        est_step_s = t_attn * (w.Lq / attn_rows) * calls + t_compress * w.n_layers + t_retrieve
+        flops_step = 4.0 * w.Lq * self.lkv * 128 * w.n_heads * calls
+        return {"value": flops_step / est_step_s / 1e12, "unit": UNIT, "cores": self.threads, "kind": "oracle",
+                "sample": (f"{attn_rows} of {w.Lq} query rows of one attention call over {self.lkv} KV tokens "
+                           f"({t_attn:.2f} s), one compression problem ({t_compress:.2f} s), one retrieval over "
+                           f"{w.pool_chunks} poses ({t_retrieve * 1e3:.2f} ms); scaled to {calls} calls + "
+                           f"{w.n_layers} problems per step"),
+                "est_step_ms": est_step_s * 1e3, "sample_seconds": t_attn + t_compress + t_retrieve}
+
+
+def run_reference(args, w: wi.Workload):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    sample = OracleSample(w)
+    rows = max(1, args.oracle_rows // 4)
+    times, last = [], None
+    for i in range(args.warmup + args.steps):
+        last = sample.run(rows)
+        if i >= args.warmup:
+            times.append(last)
+    value = statistics.mean(t["value"] for t in times)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": statistics.mean(t["est_step_ms"] for t in times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "note": "CPU oracle on a bounded sample per step, scaled to one chunk step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0, "sample_seconds": statistics.mean(t["sample_seconds"] for t in times)}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ main
+def run_ours(args, w: wi.Workload):
+    import torch
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2605_22718_b200.build import build_all
+    if rank == 0:
+        build_all()
+    barrier()
+    peaks = load_peaks()
+    bench = ChunkStepBench(w, local_rank, e2e=not args.no_e2e)
+    dev = bench.dev
+    for _ in range(args.warmup):
+        bench.step()
+    torch.cuda.synchronize(dev)
+    sampler = ClockSampler(local_rank)
+    launches0 = bench.kv.launch_count()
+    if rank == 0:
+        sampler.start()
+    ms = bench.time_steps(args.steps, host_io=False)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = bench.kv.launch_count() - launches0
+    ms = max_over_ranks(ms, dev)
+    attn_ms = [a.elapsed_time(b) for a, b in bench.attn_events]
+    st, flags = bench.kv.poll_status()
+    if st != 0:
+        raise RuntimeError(f"device status after the timed region: {st} flags {flags}")
+    e2e = None
+    if not args.no_e2e:
+        for _ in range(1):
+            bench.step(host_io=True)
+        ms_e2e = max_over_ranks(bench.time_steps(args.steps, host_io=True), dev)
+    calls = bench.attention_calls_per_step()
+    flops_call = bench.attention_flops_per_call()
+    flops_step = flops_call * calls
+    ms_per_step = ms / args.steps
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    if not args.no_e2e:
+        h2d = bench.hQ.numel() * 2 + bench.hcurK.numel() * 2 + bench.hcurV.numel() * 2
+        d2h = bench.hO.numel() * 2
+        e2e = {"value": world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps}
+    if rank != 0:
+        return
+    attn_launch_ms = statistics.mean(attn_ms) / calls
+    achieved = flops_call / (attn_launch_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    comp_bytes = 7.5 * w.T * w.D * 2 * w.n_layers
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": w.name, "layers": w.n_layers, "denoise_steps": w.denoise_steps, "heads": w.n_heads,
+                   "tokens_per_frame": w.T, "lq": w.Lq, "lkv": w.Lkv, "pool_chunks": w.pool_chunks, "k": w.k,
+                   "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "1gpu"},
+        "chunk_step_ms": ms_per_step,
+        "attention": {"calls_per_step": calls, "flops_per_call": flops_call, "ms_per_call": attn_launch_ms,
+                      "tflops": achieved, "share_of_step": statistics.mean(attn_ms) / ms_per_step},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "memory_attention_kernel"},
+        "compress_append_bytes_per_step": comp_bytes,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+    }
+    if not args.no_cpu_baseline:
+        cb = OracleSample(w).run(args.oracle_rows)
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(wi.WORKLOADS))
+    ap.add_argument("--oracle-rows", type=int, default=1024)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    w = wi.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
