@@ -355,7 +355,11 @@ def run_ours(args, w: wi.Workload):
     launches0 = bench.kv.launch_count()
     if rank == 0:
         sampler.start()
+    if args.profiler_range:   # lets `ncu --profile-from-start off` see the timed steps only
+        torch.cuda.cudart().cudaProfilerStart()
     ms = bench.time_steps(args.steps, host_io=False)
+    if args.profiler_range:
+        torch.cuda.cudart().cudaProfilerStop()
     clocks = sampler.stop() if rank == 0 else None
     launches = bench.kv.launch_count() - launches0
     ms = max_over_ranks(ms, dev)
@@ -415,6 +419,7 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(wi.WORKLOADS))
     ap.add_argument("--oracle-rows", type=int, default=1024)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profiler-range", action="store_true", help="bracket the timed steps with cudaProfilerStart/Stop")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
