@@ -1,0 +1,45 @@
+"""bench.py's multi-rank plumbing on CPU (gloo, world size 2) and its reference arm."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    sys.path.insert(0, ROOT)
+    import bench
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    bench.barrier()
+    ms = bench.max_over_ranks(10.0 + 5.0 * rank, torch.device("cpu"))
+    out[rank] = ms
+    bench.barrier()
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_and_barrier_gloo():
+    world = 2
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_worker, args=(world, 29591, out), nprocs=world, join=True)
+        assert dict(out) == {0: 15.0, 1: 15.0}          # every rank sees the slowest rank's time
+
+
+def test_reference_arm_prints_one_json_line_on_rank_0_only():
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg0", "--steps", "1",
+           "--warmup", "0"]
+    out = subprocess.run(cmd, capture_output=True, text=True, check=True).stdout.strip().splitlines()
+    assert len(out) == 1
+    line = json.loads(out[0])
+    assert line["impl"] == "reference" and line["unit"] == "TFLOP/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["gpu_launches"] == 0
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    out = subprocess.run(cmd, capture_output=True, text=True, check=True, env=env).stdout.strip()
+    assert out == ""
