@@ -124,11 +124,12 @@ def barrier():
 class ChunkStepBench:
     """Holds the pool, the per-layer window buffers and rotating inputs of one workload, and runs chunk steps."""
 
-    def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True):
+    def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True, kv_splits: int = 0):
         import torch
         from paper_2605_22718_b200 import WorldKV
         from wkinputs import device as wd
         self.torch, self.wd, self.w = torch, wd, w
+        self.kv_splits = kv_splits
         self.dev = torch.device("cuda", device_index)
         torch.cuda.set_device(self.dev)
         L, H, T, D = w.n_layers, w.n_heads, w.T, w.D
@@ -226,7 +227,7 @@ class ChunkStepBench:
                 segs = [(self.curK[l], self.curV[l])]
                 if w.window_frames > 0:
                     segs.append((self.winK[l], self.winV[l]))
-                kv.memory_attention(l, self.Q[l, s], segs, self.slots, n, O=self.O[l, s])
+                kv.memory_attention(l, self.Q[l, s], segs, self.slots, n, O=self.O[l, s], kv_splits=self.kv_splits)
         if record_attention_events:
             e1.record()
             self.attn_events.append((e0, e1))
@@ -346,7 +347,7 @@ def run_ours(args, w: wi.Workload):
         build_all()
     barrier()
     peaks = load_peaks()
-    bench = ChunkStepBench(w, local_rank, e2e=not args.no_e2e)
+    bench = ChunkStepBench(w, local_rank, e2e=not args.no_e2e, kv_splits=args.kv_splits)
     dev = bench.dev
     for _ in range(args.warmup):
         bench.step()
@@ -418,6 +419,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(wi.WORKLOADS))
     ap.add_argument("--oracle-rows", type=int, default=1024)
+    ap.add_argument("--kv-splits", type=int, default=0, help="wk_memory_attention's kv_splits argument (0 = default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profiler-range", action="store_true", help="bracket the timed steps with cudaProfilerStart/Stop")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -143,7 +143,9 @@ typedef struct {
  *   slots_dev [n_slots] int32 in device memory (e.g. wk_retrieve's output); an entry that is -1 is
  *             skipped silently, any other out-of-range or invalid entry is skipped and sets
  *             WK_DEV_BAD_SLOT; a slot listed twice is attended twice
- *   kv_splits 0 = choose automatically; otherwise 1 .. max_splits
+ *   kv_splits 0 = cut the (head, 256-row query block) x KV-tile space into one equal range per SM (default);
+ *             s in 1 .. max_splits = cut every block's KV range into s parts; -g = cut the whole space into g
+ *             equal ranges (g CTAs; needs 2 g partial slots, see wk_scratch_bytes)
  * Errors: WK_ERR_SHAPE (lq > max_lq, n_slots > max_k, n_segs > max_dense_segments, kv_splits > max_splits),
  * WK_ERR_ARG (no KV at all: n_segs = 0 and n_slots = 0), WK_ERR_UNBOUND, WK_ERR_CUDA. */
 wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, const wk_dense_seg* segs_host,

@@ -211,7 +211,7 @@ class WorldKV:
         st = self.lib.wk_memory_attention(self.ctx, layer, Q.data_ptr(), lq, arr, len(segs), _ptr(slots), n_slots,
                                           O.data_ptr(), _ptr(lse_out), kv_splits, _stream(stream))
         if st != WK_OK:
-            raise WkError(st, "wk_memory_attention")
+            raise WkError(st, f"wk_memory_attention (last CUDA error {self.last_cuda_error()})")
         return O
 
     # ---- status -------------------------------------------------------------------------------

@@ -36,10 +36,9 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   s.part_off = off;  off += align_up(B * s.anchor_parts * D * sizeof(double), 256);
   s.cnt_off = off;   off += align_up(B * sizeof(uint32_t), 256);
   s.dist_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * 2 * sizeof(double), 256);
-  const size_t lqp = align_up(static_cast<size_t>(max_lq > 0 ? max_lq : 1), 2 * kTileQ);
-  const size_t sp = static_cast<size_t>(max_splits > 1 ? max_splits : 0);
-  s.opart_off = off;   off += align_up(sp * c.n_heads * lqp * kHeadDim * sizeof(float), 256);
-  s.lsepart_off = off; off += align_up(sp * c.n_heads * lqp * sizeof(float), 256);
+  const size_t slots = static_cast<size_t>(attention_partial_slots(c.n_heads, max_lq > 0 ? max_lq : 1, max_splits));
+  s.opart_off = off;   off += align_up(slots * 2 * kTileQ * kHeadDim * sizeof(float), 256);
+  s.lsepart_off = off; off += align_up(slots * 2 * kTileQ * sizeof(float), 256);
   s.total = off;
   return s;
 }
@@ -315,7 +314,7 @@ wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t
   if (!aligned16(Q) || !aligned16(O)) return WK_ERR_ARG;
   if (layer < 0 || layer >= ctx->cfg.n_layers) return WK_ERR_SHAPE;
   if (lq > ctx->max_lq || n_slots > ctx->cfg.max_k || n_segs > ctx->cfg.max_dense_segments) return WK_ERR_SHAPE;
-  if (kv_splits < 0 || kv_splits > (ctx->max_splits > 1 ? ctx->max_splits : 1)) return WK_ERR_SHAPE;
+  if (kv_splits > (ctx->max_splits > 1 ? ctx->max_splits : 1)) return WK_ERR_SHAPE;
   for (int i = 0; i < n_segs; ++i) {
     if (!segs_host[i].K || !segs_host[i].V || segs_host[i].n_tokens < 1) return WK_ERR_ARG;
     if (!aligned16(segs_host[i].K) || !aligned16(segs_host[i].V)) return WK_ERR_ARG;

@@ -2,7 +2,10 @@
 // [dense segments ..., retrieved pool slots ...] of one layer.  O = softmax(scale Q K^T) V per head.
 //
 // Flash-style kernel on the 5th-generation tensor cores:
-//   * one CTA owns two 128-row Q tiles of one head (256 query rows) and a contiguous range of KV tiles;
+//   * a work unit is (head, 256 query rows = two 128-row Q tiles); the flat space unit x KV tile is cut into equal
+//     contiguous ranges, one per CTA (one CTA per SM by default), so every SM gets the same amount of work.  A range
+//     that covers a whole unit writes bf16 output directly; otherwise it writes a normalised fp32 partial plus its
+//     log-sum-exp and combine_kernel merges the (at most three) pieces of that unit;
 //   * K/V tiles (128 rows x 128 columns of one head, bf16) are fetched by TMA straight from where they lie:
 //     a dense segment (2-D tensor map per segment) or a pool slot (3-D tensor map [layer*slot][row][col]; the
 //     slot id is read from device memory, so the retrieval result never visits the host).  Rows past the end
@@ -11,9 +14,10 @@
 //     memory: S0, S1, O0, O1 fill all 512 columns; P (bf16) overwrites S in place and is the A operand of
 //     the P V product directly from tensor memory;
 //   * warp roles: warps 0-3 / 4-7 = softmax of Q tile 0 / 1 (one thread per row, online softmax in fp32 in
-//     the exp2 domain, running maximum updated lazily), warp 8 = MMA issue, warp 9 = TMA producer;
-//   * with kv splits, each CTA writes normalised fp32 partials + log-sum-exp and a combine kernel merges them.
+//     the exp2 domain, running maximum updated lazily), warp 8 = MMA issue, warp 9 = TMA producer.
 // Every wait is bounded; a wait that runs out sets WK_DEV_TIMEOUT, the CTA drains and frees its tensor memory.
+#include <stdlib.h>
+
 #include "ptx_sm100.cuh"
 #include "wk_internal.cuh"
 
@@ -29,6 +33,9 @@ constexpr uint32_t kTileBytes = 2 * kHalfTileBytes; // 128 x 128 bf16
 constexpr int kStages = 2;
 constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + 2 * kStages * kTileBytes;   // align slack + Q0,Q1 + K,V stages
 constexpr float kRescaleThreshold = 8.0f;           // log2 units: P stays <= 2^8 between maximum updates
+constexpr int kPairRows = 2 * kTileQ;
+constexpr int kDefaultPoly = 0;
+constexpr int kMaxPieces = 32;                      // most ranges one unit may be cut into
 
 struct AttnParams {
   CUtensorMap tm_q;
@@ -40,56 +47,108 @@ struct AttnParams {
   const int32_t* slots;
   const int32_t* valid;
   int n_slots, pool_slots, layer, C, tiles_per_slot;
-  int n_tiles, splits;
-  int lq, lq_pad, H;
+  int n_tiles, n_qpairs, n_units;
+  int lq, H;
   float scale_log2;
   __nv_bfloat16* O;
   float* lse;
-  float* opart;
-  float* lsepart;
+  float* opart;     // [2 * gridDim.x][256][128] fp32
+  float* lsepart;   // [2 * gridDim.x][256]
   uint32_t* status;
 };
+
+__device__ __forceinline__ int64_t range_start(const AttnParams& p, int c, int G) {
+  return static_cast<int64_t>(c) * p.n_units * p.n_tiles / G;
+}
 
 struct TileInfo {
   int seg;    // >= 0: dense segment index; -1: pool
   int row0;
   int z;
-  int nv;     // valid rows, 0 = skip
+  int nv;     // valid rows (> 0)
 };
 
-__device__ __forceinline__ TileInfo kv_tile(const AttnParams& p, int t, bool report) {
-  TileInfo ti;
-  if (t < p.n_dense_tiles) {
-    int i = 0;
-    while (i + 1 < p.n_segs && t >= p.seg_tile_prefix[i + 1]) ++i;
-    ti.seg = i;
-    ti.row0 = (t - p.seg_tile_prefix[i]) * kTileKV;
-    ti.z = 0;
-    ti.nv = min(kTileKV, p.seg_rows[i] - ti.row0);
-  } else {
-    const int u = t - p.n_dense_tiles;
-    const int si = u / p.tiles_per_slot, r = u - si * p.tiles_per_slot;
+// Walks the effective KV tiles of [tb, te): dense segments first, then pool slots; stale or -1 slots are skipped.
+struct TileIter {
+  int t, te, seg, si, r, z;
+  bool slot_ok;
+  __device__ __forceinline__ void load_slot(const AttnParams& p, bool report) {
     const int slot = __ldg(p.slots + si);
-    ti.seg = -1;
-    ti.row0 = r * kTileKV;
     bool ok = slot >= 0 && slot < p.pool_slots;
     if (ok) ok = __ldg(p.valid + slot) != 0;
-    if (!ok) {
-      if (report && slot != -1) atomicOr(p.status, WK_DEV_BAD_SLOT);   // never dereferenced
-      ti.nv = 0;
-      ti.z = 0;
-    } else {
-      ti.z = p.layer * p.pool_slots + slot;
-      ti.nv = min(kTileKV, p.C - ti.row0);
+    if (!ok && report && slot != -1) atomicOr(p.status, WK_DEV_BAD_SLOT);   // never dereferenced
+    slot_ok = ok;
+    z = ok ? p.layer * p.pool_slots + slot : 0;
+  }
+  __device__ __forceinline__ void init(const AttnParams& p, int tb, int te_, bool report) {
+    t = tb;
+    te = te_;
+    seg = 0;
+    si = -1;
+    r = 0;
+    slot_ok = false;
+    z = 0;
+    if (t >= p.n_dense_tiles && t < te) {
+      const int u = t - p.n_dense_tiles;
+      si = u / p.tiles_per_slot;
+      r = u - si * p.tiles_per_slot;
+      load_slot(p, report);
     }
   }
-  return ti;
-}
+  __device__ __forceinline__ bool next(const AttnParams& p, TileInfo& ti, bool report) {
+    while (t < te) {
+      if (t < p.n_dense_tiles) {
+        while (seg + 1 < p.n_segs && t >= p.seg_tile_prefix[seg + 1]) ++seg;
+        ti.seg = seg;
+        ti.row0 = (t - p.seg_tile_prefix[seg]) * kTileKV;
+        ti.z = 0;
+        ti.nv = min(kTileKV, p.seg_rows[seg] - ti.row0);
+        ++t;
+        return true;
+      }
+      if (si < 0) {   // first pool tile of this range
+        si = 0;
+        r = 0;
+        load_slot(p, report);
+      }
+      const bool ok = slot_ok;
+      ti.seg = -1;
+      ti.row0 = r * kTileKV;
+      ti.z = z;
+      ti.nv = min(kTileKV, p.C - ti.row0);
+      ++t;
+      if (++r == p.tiles_per_slot) {
+        r = 0;
+        ++si;
+        if (t < te) load_slot(p, report);
+      }
+      if (ok) return true;
+    }
+    return false;
+  }
+};
+
+#ifdef WK_ATTN_PROFILE
+// Stage timers for one designated thread per role of CTA 0: clock deltas (in 16-clock units) are added into the words
+// after the status word.  Built only for profiling runs; the product build has none of this.
+#define WK_PROF_DECL long long prof_t = clock64();
+#define WK_PROF(slot, cond)                                                              \
+  do {                                                                                   \
+    if (cond) {                                                                          \
+      const long long now__ = clock64();                                                 \
+      atomicAdd(p.status + 8 + (slot), static_cast<uint32_t>((now__ - prof_t) >> 4));    \
+      prof_t = now__;                                                                    \
+    }                                                                                    \
+  } while (0)
+#else
+#define WK_PROF_DECL
+#define WK_PROF(slot, cond)
+#endif
 
 struct __align__(8) Barriers {
-  uint64_t q_full;
+  uint64_t q_full, q_empty;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], p_full[2], o_done[2];
+  uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
 };
 
 // Bounded wait that also gives up when another role has already aborted.
@@ -104,6 +163,81 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t* bar, uint32_t parity, vo
   return false;
 }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x for a pair of fp32 values in [-126, 9] on the FMA/ALU pipes instead of the MUFU: x = n + f with n = round(x)
+// (magic-number rounding), 2^f by a cubic on [-0.5, 0.5] (relative error 2e-4, ten times below the bf16 rounding
+// P receives anyway), n added into the exponent field.
+__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& p0, float& p1) {
+  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+  const uint64_t x = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const uint64_t xr = add_f32x2(x, magic);                                   // low mantissa bits hold round(x)
+  const uint64_t n = add_f32x2(xr, neg_magic);
+  const uint64_t f = fma_f32x2(n, pack_f32x2(-1.f, -1.f), x);
+  uint64_t q = fma_f32x2(f, pack_f32x2(0.053027522f, 0.053027522f), pack_f32x2(0.24221395f, 0.24221395f));
+  q = fma_f32x2(q, f, pack_f32x2(0.69357258f, 0.69357258f));
+  q = fma_f32x2(q, f, pack_f32x2(0.99995905f, 0.99995905f));
+  float q0, q1, r0, r1;
+  unpack_f32x2(q, q0, q1);
+  unpack_f32x2(xr, r0, r1);
+  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(r0) << 23));
+  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
+}
+
+// One piece of work: unit u, KV tiles [tb, te), and where its result goes.
+struct Piece {
+  int h, q0, tb, te, slot;   // slot < 0: the piece covers the whole unit -> direct output
+  bool has_q1;
+};
+struct PieceWalker {
+  int64_t pos, end, start;
+  int cta;
+  __device__ __forceinline__ void init(const AttnParams& p) {
+    cta = blockIdx.x;
+    start = range_start(p, cta, gridDim.x);
+    end = range_start(p, cta + 1, gridDim.x);
+    pos = start;
+  }
+  __device__ __forceinline__ bool next(const AttnParams& p, Piece& pc) {
+    if (pos >= end) return false;
+    const int u = static_cast<int>(pos / p.n_tiles);
+    pc.tb = static_cast<int>(pos - static_cast<int64_t>(u) * p.n_tiles);
+    const int64_t room = end - pos;
+    pc.te = static_cast<int>(min(static_cast<int64_t>(p.n_tiles), pc.tb + room));
+    pc.h = u / p.n_qpairs;
+    pc.q0 = (u - pc.h * p.n_qpairs) * kPairRows;
+    pc.has_q1 = pc.q0 + kTileQ < p.lq;
+    const bool full = pc.tb == 0 && pc.te == p.n_tiles;
+    pc.slot = full ? -1 : 2 * cta + (pos == start ? 0 : 1);
+    pos += pc.te - pc.tb;
+    return true;
+  }
+};
+
+// NPOLY of every four element pairs take the polynomial exp2, the rest the MUFU.
+template <int NPOLY>
 __global__ void __launch_bounds__(kThreads, 1)
 memory_attention_kernel(const __grid_constant__ AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -116,20 +250,17 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
   __shared__ volatile uint32_t s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qpair = blockIdx.x, h = blockIdx.y, split = blockIdx.z;
-  const int q0 = qpair * 2 * kTileQ;
-  const bool has_q1 = q0 + kTileQ < p.lq;
-  const int t0 = static_cast<int>(static_cast<int64_t>(p.n_tiles) * split / p.splits);
-  const int t1 = static_cast<int>(static_cast<int64_t>(p.n_tiles) * (split + 1) / p.splits);
 
   if (tid == 0) {
     mbar_init(&bars.q_full, 1);
+    mbar_init(&bars.q_empty, 1);
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1);
       mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.s_full[i], 1); mbar_init(&bars.p_full[i], 128); mbar_init(&bars.o_done[i], 1);
+      mbar_init(&bars.o_free[i], 128);
     }
     s_abort = 0;
     fence_mbar_init();
@@ -146,40 +277,48 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
   if (warp == kTmaWarp) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      mbar_expect_tx(&bars.q_full, 2 * kTileBytes);
-      for (int i = 0; i < 2; ++i)
-        for (int half = 0; half < 2; ++half)
-          tma_load_2d(sQ + i * kTileBytes + half * kHalfTileBytes, &p.tm_q, &bars.q_full, h * kHeadDim + half * 64,
-                      q0 + i * kTileQ);
-      int j = 0;
-      const bool report = (blockIdx.x == 0 && blockIdx.y == 0);
-      for (int t = t0; t < t1; ++t) {
-        const TileInfo ti = kv_tile(p, t, report);
-        if (ti.nv == 0) continue;
-        const int st = j % kStages;
-        const uint32_t ph = (j / kStages) & 1;
-        const int x = h * kHeadDim;
-        if (!wait_or_abort(&bars.k_empty[st], ph ^ 1, &s_abort, p.status)) break;
-        mbar_expect_tx(&bars.k_full[st], kTileBytes);
-        uint8_t* dk = sK + st * kTileBytes;
-        if (ti.seg >= 0) {
-          tma_load_2d(dk, &p.tm_kd[ti.seg], &bars.k_full[st], x, ti.row0);
-          tma_load_2d(dk + kHalfTileBytes, &p.tm_kd[ti.seg], &bars.k_full[st], x + 64, ti.row0);
-        } else {
-          tma_load_3d(dk, &p.tm_kpool, &bars.k_full[st], x, ti.row0, ti.z);
-          tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[st], x + 64, ti.row0, ti.z);
+      PieceWalker walk;
+      walk.init(p);
+      Piece pc;
+      uint32_t jk = 0, n = 0;
+      bool ok = true;
+      while (ok && walk.next(p, pc)) {
+        if (!(ok = wait_or_abort(&bars.q_empty, (n & 1) ^ 1, &s_abort, p.status))) break;
+        mbar_expect_tx(&bars.q_full, 2 * kTileBytes);
+        for (int i = 0; i < 2; ++i)
+          for (int half = 0; half < 2; ++half)
+            tma_load_2d(sQ + i * kTileBytes + half * kHalfTileBytes, &p.tm_q, &bars.q_full, pc.h * kHeadDim + half * 64,
+                        pc.q0 + i * kTileQ);
+        TileIter it;
+        it.init(p, pc.tb, pc.te, true);
+        TileInfo ti;
+        const int x = pc.h * kHeadDim;
+        while (it.next(p, ti, true)) {
+          const int st = jk % kStages;
+          const uint32_t ph = (jk / kStages) & 1;
+          if (!(ok = wait_or_abort(&bars.k_empty[st], ph ^ 1, &s_abort, p.status))) break;
+          mbar_expect_tx(&bars.k_full[st], kTileBytes);
+          uint8_t* dk = sK + st * kTileBytes;
+          if (ti.seg >= 0) {
+            tma_load_2d(dk, &p.tm_kd[ti.seg], &bars.k_full[st], x, ti.row0);
+            tma_load_2d(dk + kHalfTileBytes, &p.tm_kd[ti.seg], &bars.k_full[st], x + 64, ti.row0);
+          } else {
+            tma_load_3d(dk, &p.tm_kpool, &bars.k_full[st], x, ti.row0, ti.z);
+            tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[st], x + 64, ti.row0, ti.z);
+          }
+          if (!(ok = wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status))) break;
+          mbar_expect_tx(&bars.v_full[st], kTileBytes);
+          uint8_t* dv = sV + st * kTileBytes;
+          if (ti.seg >= 0) {
+            tma_load_2d(dv, &p.tm_vd[ti.seg], &bars.v_full[st], x, ti.row0);
+            tma_load_2d(dv + kHalfTileBytes, &p.tm_vd[ti.seg], &bars.v_full[st], x + 64, ti.row0);
+          } else {
+            tma_load_3d(dv, &p.tm_vpool, &bars.v_full[st], x, ti.row0, ti.z);
+            tma_load_3d(dv + kHalfTileBytes, &p.tm_vpool, &bars.v_full[st], x + 64, ti.row0, ti.z);
+          }
+          ++jk;
         }
-        if (!wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status)) break;
-        mbar_expect_tx(&bars.v_full[st], kTileBytes);
-        uint8_t* dv = sV + st * kTileBytes;
-        if (ti.seg >= 0) {
-          tma_load_2d(dv, &p.tm_vd[ti.seg], &bars.v_full[st], x, ti.row0);
-          tma_load_2d(dv + kHalfTileBytes, &p.tm_vd[ti.seg], &bars.v_full[st], x + 64, ti.row0);
-        } else {
-          tma_load_3d(dv, &p.tm_vpool, &bars.v_full[st], x, ti.row0, ti.z);
-          tma_load_3d(dv + kHalfTileBytes, &p.tm_vpool, &bars.v_full[st], x + 64, ti.row0, ti.z);
-        }
-        ++j;
+        ++n;
       }
       // Do not leave while copies may still be landing in shared memory: wait (bounded) for the loads issued last.
       if (s_abort) {
@@ -197,62 +336,108 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
       const uint32_t idesc_pv = idesc_bf16_f32(128, 128, 0, 1);
       const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
-      // number of tiles this CTA really processes
-      int n_eff = 0;
-      for (int t = t0; t < t1; ++t) n_eff += (kv_tile(p, t, false).nv != 0);
+      // descriptor low words of the tile bases; a K = 16 step advances them by a constant
+      const uint32_t hi = smem_desc_hi_sw128(1024);
+      const uint32_t q_lo0 = smem_desc_lo(aQ, 16), q_lo1 = smem_desc_lo(aQ + kTileBytes, 16);
+      const uint32_t k_lo0 = smem_desc_lo(aK, 16), v_lo0 = smem_desc_lo(aV, kHalfTileBytes);
       auto issue_s = [&](int i, int st) {
         const uint32_t d = tmem + i * 128;
+        const uint32_t a_lo = i ? q_lo1 : q_lo0, b_lo = k_lo0 + st * (kTileBytes >> 4);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * kHalfTileBytes + (k & 3) * 32;
-          mma_ss(d, smem_desc_sw128(aQ + i * kTileBytes + off, 16, 1024), smem_desc_sw128(aK + st * kTileBytes + off, 16, 1024),
-                 idesc_qk, k > 0);
+          const uint32_t off = (k >> 2) * (kHalfTileBytes >> 4) + (k & 3) * 2;   // 32 bytes per step inside a 128-byte row
+          mma_ss_lohi(d, a_lo + off, b_lo + off, hi, idesc_qk, k > 0);
         }
       };
       auto issue_pv = [&](int i, int st, bool accumulate) {
         const uint32_t d = tmem + 256 + i * 128;
+        const uint32_t b_lo = v_lo0 + st * (kTileBytes >> 4);
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          // A = P from tensor memory (bf16 pairs, 8 columns per K = 16 step); B = V, rows = K dimension, MN-major
-          mma_ts(d, tmem + i * 128 + k * 8, smem_desc_sw128(aV + st * kTileBytes + k * 2048, kHalfTileBytes, 1024), idesc_pv,
-                 accumulate || k > 0);
+          // A = P from tensor memory (bf16 pairs, 8 columns per K = 16 step); B = V, rows = K dimension, MN-major:
+          // 16 rows of 128 bytes = 2048 bytes per step
+          mma_ts_lohi(d, tmem + i * 128 + k * 8, b_lo + k * 128, hi, idesc_pv, (accumulate || k > 0) ? 1u : 0u);
         }
       };
-      bool ok = n_eff > 0 && wait_or_abort(&bars.q_full, 0, &s_abort, p.status);
-      if (ok) ok = wait_or_abort(&bars.k_full[0], 0, &s_abort, p.status);
-      if (ok) {
-        tc_fence_after();
-        issue_s(0, 0);
-        mma_commit(&bars.s_full[0]);
-        if (has_q1) { issue_s(1, 0); mma_commit(&bars.s_full[1]); }
-        mma_commit(&bars.k_empty[0]);
-      }
-      for (int j = 0; ok && j < n_eff; ++j) {
-        const int st = j % kStages, stn = (j + 1) % kStages;
-        const uint32_t ph = (j / kStages) & 1, phn = ((j + 1) / kStages) & 1;
-        const bool more = j + 1 < n_eff;
-        if (!(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
-        if (!(ok = wait_or_abort(&bars.p_full[0], j & 1, &s_abort, p.status))) break;
-        tc_fence_after();
-        issue_pv(0, st, j > 0);
-        mma_commit(&bars.o_done[0]);
-        if (more) {
-          if (!(ok = wait_or_abort(&bars.k_full[stn], phn, &s_abort, p.status))) break;
+      PieceWalker walk;
+      walk.init(p);
+      Piece pc;
+      uint32_t g0 = 0, g1 = 0, n = 0;   // running tile counts of the two Q tiles, running piece count
+      uint32_t e0 = 0, e1 = 0;          // pieces in which Q tile 0 / 1 produced output so far
+      WK_PROF_DECL
+      bool ok = true;
+      while (ok && walk.next(p, pc)) {
+        int n_eff = 0;
+        {
+          TileIter it;
+          it.init(p, pc.tb, pc.te, false);
+          TileInfo ti;
+          while (it.next(p, ti, false)) ++n_eff;
+        }
+        const bool q1 = pc.has_q1;
+        if (!(ok = wait_or_abort(&bars.q_full, n & 1, &s_abort, p.status))) break;
+        ++n;
+        if (n_eff == 0) {
+          mbar_arrive(&bars.q_empty);
+          continue;
+        }
+        // O0 / O1 are about to be overwritten: the epilogue of the last piece that used them must have read them.
+        // o_free[i] completes once per piece in which warpgroup i ran an epilogue, so neither side can run two
+        // phases ahead of the other (a parity wait cannot tell phase n from phase n + 2).
+        if (e0 > 0 && !(ok = wait_or_abort(&bars.o_free[0], (e0 - 1) & 1, &s_abort, p.status))) break;
+        ++e0;
+        if (q1) {
+          if (e1 > 0 && !(ok = wait_or_abort(&bars.o_free[1], (e1 - 1) & 1, &s_abort, p.status))) break;
+          ++e1;
+        }
+        {
+          const int st = g0 % kStages;
+          if (!(ok = wait_or_abort(&bars.k_full[st], (g0 / kStages) & 1, &s_abort, p.status))) break;
           tc_fence_after();
-          issue_s(0, stn);
+          issue_s(0, st);
           mma_commit(&bars.s_full[0]);
+          if (q1) { issue_s(1, st); mma_commit(&bars.s_full[1]); }
+          mma_commit(&bars.k_empty[st]);
+          if (n_eff == 1) mma_commit(&bars.q_empty);
         }
-        if (has_q1) {
-          if (!(ok = wait_or_abort(&bars.p_full[1], j & 1, &s_abort, p.status))) break;
+        for (int j = 0; j < n_eff; ++j) {
+          const uint32_t g = g0 + j;
+          const int st = g % kStages, stn = (g + 1) % kStages;
+          const uint32_t ph = (g / kStages) & 1, phn = ((g + 1) / kStages) & 1;
+          const bool more = j + 1 < n_eff;
+          WK_PROF(10, blockIdx.x == 0);
+          if (!(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
+          WK_PROF(11, blockIdx.x == 0);
+          if (!(ok = wait_or_abort(&bars.p_full[0], g & 1, &s_abort, p.status))) break;
+          WK_PROF(12, blockIdx.x == 0);
           tc_fence_after();
-          issue_pv(1, st, j > 0);
-          mma_commit(&bars.o_done[1]);
+          issue_pv(0, st, j > 0);
+          mma_commit(&bars.o_done[0]);
+          if (more) {
+            WK_PROF(13, blockIdx.x == 0);
+            if (!(ok = wait_or_abort(&bars.k_full[stn], phn, &s_abort, p.status))) break;
+            WK_PROF(14, blockIdx.x == 0);
+            tc_fence_after();
+            issue_s(0, stn);
+            mma_commit(&bars.s_full[0]);
+          }
+          if (q1) {
+            WK_PROF(15, blockIdx.x == 0);
+            if (!(ok = wait_or_abort(&bars.p_full[1], (g1 + j) & 1, &s_abort, p.status))) break;
+            WK_PROF(16, blockIdx.x == 0);
+            tc_fence_after();
+            issue_pv(1, st, j > 0);
+            mma_commit(&bars.o_done[1]);
+          }
+          mma_commit(&bars.v_empty[st]);
+          if (more) {
+            if (q1) { issue_s(1, stn); mma_commit(&bars.s_full[1]); }
+            mma_commit(&bars.k_empty[stn]);
+            if (j + 2 == n_eff) mma_commit(&bars.q_empty);   // the last Q K^T of this piece has been issued
+          }
         }
-        mma_commit(&bars.v_empty[st]);
-        if (more) {
-          if (has_q1) { issue_s(1, stn); mma_commit(&bars.s_full[1]); }
-          mma_commit(&bars.k_empty[stn]);
-        }
+        g0 += n_eff;
+        if (q1) g1 += n_eff;
       }
     }
   } else {
@@ -262,125 +447,166 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t tS = tmem + lane_base + wg * 128;
     const uint32_t tO = tmem + lane_base + 256 + wg * 128;
-    const bool active = (wg == 0) || has_q1;
-    float m_used = -INFINITY, l = 0.f;
-    int j = 0;
+    PieceWalker walk;
+    walk.init(p);
+    Piece pc;
+    uint32_t g = 0;   // running tile count of this warpgroup
     bool ok = true;
-    if (active) {
-      for (int t = t0; t < t1 && ok; ++t) {
-        const int nv = kv_tile(p, t, false).nv;
-        if (nv == 0) continue;
-        if (!(ok = wait_or_abort(&bars.s_full[wg], j & 1, &s_abort, p.status))) break;
-        tc_fence_after();
-        float s[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          tmem_ld_x32(tS + c * 32, r);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
-        }
-        tc_wait_ld();
-        float mx = -INFINITY;
-        if (nv == kTileKV) {
-#pragma unroll
-          for (int i = 0; i < 128; ++i) mx = fmaxf(mx, s[i]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 128; ++i) {
-            s[i] = i < nv ? s[i] : -INFINITY;       // rows past the end of the segment were zero-filled by TMA
-            mx = fmaxf(mx, s[i]);
-          }
-        }
-        const float m_new = fmaxf(m_used, mx * p.scale_log2);
-        float alpha = 1.f;
-        bool rescale = false;
-        if (m_new > m_used + kRescaleThreshold) {    // also true on the first tile (m_used = -inf)
-          alpha = ex2_approx(m_used - m_new);
-          m_used = m_new;
-          rescale = j > 0;
-        }
-        l *= alpha;
-        const float neg_m = -m_used;
-        float sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float p0 = ex2_approx(fmaf(s[c * 32 + 2 * i], p.scale_log2, neg_m));
-            const float p1 = ex2_approx(fmaf(s[c * 32 + 2 * i + 1], p.scale_log2, neg_m));
-            sum += p0 + p1;
-            pk[i] = pack_bf16x2(p0, p1);
-          }
-          tmem_st_x16(tS + c * 16, pk);
-        }
-        l += sum;
-        if (__any_sync(0xffffffffu, rescale)) {
-          // the previous P V product must have landed before O is touched
-          if (!(ok = wait_or_abort(&bars.o_done[wg], (j - 1) & 1, &s_abort, p.status))) break;
+    WK_PROF_DECL
+    const uint64_t scale2 = pack_f32x2(p.scale_log2, p.scale_log2);
+    while (ok && walk.next(p, pc)) {
+      const bool active = (wg == 0) || pc.has_q1;
+      float m_used = -INFINITY, l = 0.f;
+      int j = 0;
+      if (active) {
+        TileIter it;
+        it.init(p, pc.tb, pc.te, false);
+        TileInfo ti;
+        while (it.next(p, ti, false)) {
+          const int nv = ti.nv;
+          WK_PROF(0, blockIdx.x == 0 && tid == 0);
+          if (!(ok = wait_or_abort(&bars.s_full[wg], g & 1, &s_abort, p.status))) break;
+          WK_PROF(1, blockIdx.x == 0 && tid == 0);
           tc_fence_after();
+          float s[128];
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t r[32];
-            tmem_ld_x32(tO + c * 32, r);
-            tc_wait_ld();
+            tmem_ld_x32(tS + c * 32, r);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            tmem_st_x32(tO + c * 32, r);
+            for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
           }
+          tc_wait_ld();
+          WK_PROF(2, blockIdx.x == 0 && tid == 0);
+          if (nv < kTileKV) {
+#pragma unroll
+            for (int i = 0; i < 128; ++i) s[i] = i < nv ? s[i] : -INFINITY;   // zero-filled rows past the segment end
+          }
+          float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 128; i += 8) {
+            c0 = fmax3(c0, s[i], s[i + 1]);
+            c1 = fmax3(c1, s[i + 2], s[i + 3]);
+            c2 = fmax3(c2, s[i + 4], s[i + 5]);
+            c3 = fmax3(c3, s[i + 6], s[i + 7]);
+          }
+          const float mx = fmaxf(fmax3(c0, c1, c2), c3);
+          WK_PROF(3, blockIdx.x == 0 && tid == 0);
+          const float m_new = fmaxf(m_used, mx * p.scale_log2);
+          float alpha = 1.f;
+          bool rescale = false;
+          if (m_new > m_used + kRescaleThreshold) {    // also true on the first tile (m_used = -inf)
+            alpha = ex2_approx(m_used - m_new);
+            m_used = m_new;
+            rescale = j > 0;
+          }
+          l *= alpha;
+          const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
+          uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const uint64_t e = fma_f32x2(pack_f32x2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), scale2, neg_m2);
+              float e0, e1;
+              unpack_f32x2(e, e0, e1);
+              float p0, p1;
+              if ((i & 3) < NPOLY && nv == kTileKV) {
+                exp2_poly_x2(e0, e1, p0, p1);
+              } else {
+                p0 = ex2_approx(e0);
+                p1 = ex2_approx(e1);
+              }
+              const uint64_t pp = pack_f32x2(p0, p1);
+              if ((i & 3) == 0) acc0 = add_f32x2(acc0, pp);
+              else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
+              else if ((i & 3) == 2) acc2 = add_f32x2(acc2, pp);
+              else acc3 = add_f32x2(acc3, pp);
+              pk[i] = pack_bf16x2(p0, p1);
+            }
+            tmem_st_x16(tS + c * 16, pk);
+          }
+          {
+            float a, b;
+            unpack_f32x2(add_f32x2(add_f32x2(acc0, acc1), add_f32x2(acc2, acc3)), a, b);
+            l += a + b;
+          }
+          if (__any_sync(0xffffffffu, rescale)) {
+            // the previous P V product must have landed before O is touched
+            if (!(ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status))) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              uint32_t r[32];
+              tmem_ld_x32(tO + c * 32, r);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+              tmem_st_x32(tO + c * 32, r);
+            }
+          }
+          WK_PROF(4, blockIdx.x == 0 && tid == 0);
+          tc_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars.p_full[wg]);
+          WK_PROF(5, blockIdx.x == 0 && tid == 0);
+          ++j;
+          ++g;
         }
-        tc_wait_st();
-        tc_fence_before();
-        mbar_arrive(&bars.p_full[wg]);
-        ++j;
-      }
-      // ---------------------------------------------------------------- epilogue
-      const int qrow = q0 + wg * kTileQ + row;
-      if (ok && j > 0) ok = wait_or_abort(&bars.o_done[wg], (j - 1) & 1, &s_abort, p.status);
-      if (ok) {
-        tc_fence_after();
-        const float inv_l = (j > 0 && l > 0.f) ? 1.f / l : 0.f;
-        const float lse = (j > 0 && l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        // ---------------------------------------------------------------- epilogue of this piece
+        const int prow = wg * kTileQ + row;
+        const int qrow = pc.q0 + prow;
+        if (ok && j > 0) ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status);
+        if (ok) {
+          tc_fence_after();
+          const float inv_l = (j > 0 && l > 0.f) ? 1.f / l : 0.f;
+          const float lse = (j > 0 && l > 0.f) ? (m_used + log2f(l)) * 0.6931471805599453f : -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t r[32];
-          if (j > 0) {
-            tmem_ld_x32(tO + c * 32, r);
-            tc_wait_ld();
-          } else {
+          for (int c = 0; c < 4; ++c) {
+            uint32_t r[32];
+            if (j > 0) {
+              tmem_ld_x32(tO + c * 32, r);
+              tc_wait_ld();
+            } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = 0u;
+              for (int i = 0; i < 32; ++i) r[i] = 0u;
+            }
+            if (qrow < p.lq) {
+              if (pc.slot < 0) {
+                uint4* dst = reinterpret_cast<uint4*>(p.O + (static_cast<int64_t>(qrow) * p.H + pc.h) * kHeadDim + c * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                  uint4 o;
+                  o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l);
+                  o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l);
+                  o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l);
+                  o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l);
+                  dst[v] = o;
+                }
+              } else {
+                float4* dst = reinterpret_cast<float4*>(
+                    p.opart + (static_cast<int64_t>(pc.slot) * kPairRows + prow) * kHeadDim + c * 32);
+#pragma unroll
+                for (int v = 0; v < 8; ++v)
+                  dst[v] = make_float4(__uint_as_float(r[4 * v]) * inv_l, __uint_as_float(r[4 * v + 1]) * inv_l,
+                                       __uint_as_float(r[4 * v + 2]) * inv_l, __uint_as_float(r[4 * v + 3]) * inv_l);
+              }
+            }
           }
           if (qrow < p.lq) {
-            if (p.splits == 1) {
-              uint4* dst = reinterpret_cast<uint4*>(p.O + (static_cast<int64_t>(qrow) * p.H + h) * kHeadDim + c * 32);
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                uint4 o;
-                o.x = pack_bf16x2(__uint_as_float(r[8 * v + 0]) * inv_l, __uint_as_float(r[8 * v + 1]) * inv_l);
-                o.y = pack_bf16x2(__uint_as_float(r[8 * v + 2]) * inv_l, __uint_as_float(r[8 * v + 3]) * inv_l);
-                o.z = pack_bf16x2(__uint_as_float(r[8 * v + 4]) * inv_l, __uint_as_float(r[8 * v + 5]) * inv_l);
-                o.w = pack_bf16x2(__uint_as_float(r[8 * v + 6]) * inv_l, __uint_as_float(r[8 * v + 7]) * inv_l);
-                dst[v] = o;
-              }
+            if (pc.slot < 0) {
+              if (p.lse) p.lse[static_cast<int64_t>(pc.h) * p.lq + qrow] = lse;
             } else {
-              float4* dst = reinterpret_cast<float4*>(
-                  p.opart + ((static_cast<int64_t>(split) * p.H + h) * p.lq_pad + qrow) * kHeadDim + c * 32);
-#pragma unroll
-              for (int v = 0; v < 8; ++v)
-                dst[v] = make_float4(__uint_as_float(r[4 * v]) * inv_l, __uint_as_float(r[4 * v + 1]) * inv_l,
-                                     __uint_as_float(r[4 * v + 2]) * inv_l, __uint_as_float(r[4 * v + 3]) * inv_l);
+              p.lsepart[static_cast<int64_t>(pc.slot) * kPairRows + prow] = lse;
             }
           }
         }
-        if (qrow < p.lq) {
-          if (p.splits == 1) {
-            if (p.lse) p.lse[static_cast<int64_t>(h) * p.lq + qrow] = lse;
-          } else {
-            p.lsepart[(static_cast<int64_t>(split) * p.H + h) * p.lq_pad + qrow] = lse;
-          }
-        }
+      }
+      // O of this piece has been read: the next piece that uses this accumulator may overwrite it
+      if (active && j > 0) {
+        tc_fence_before();
+        mbar_arrive(&bars.o_free[wg]);
       }
     }
   }
@@ -389,19 +615,38 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
   if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-// Merge split-KV partials: O = sum_s w_s O_s / sum_s w_s with w_s = exp(lse_s - max lse).  One warp per (row, head).
+// Merge the pieces of every unit that was cut: O = sum_s w_s O_s / sum_s w_s with w_s = exp(lse_s - max lse).
+// One warp per (unit, row of the 256-row pair); units written directly by a single CTA are left alone.
 __global__ void __launch_bounds__(256)
-combine_kernel(const float* __restrict__ opart, const float* __restrict__ lsepart, int splits, int H, int lq, int lq_pad,
-               __nv_bfloat16* __restrict__ O, float* __restrict__ lse_out) {
+combine_kernel(const float* __restrict__ opart, const float* __restrict__ lsepart, int G, int n_units, int n_tiles,
+               int n_qpairs, int H, int lq, __nv_bfloat16* __restrict__ O, float* __restrict__ lse_out) {
   const int warp_global = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (warp_global >= lq * H) return;
-  const int qrow = warp_global / H, h = warp_global - qrow * H;
+  if (warp_global >= n_units * kPairRows) return;
+  const int u = warp_global / kPairRows, prow = warp_global - u * kPairRows;
+  const int h = u / n_qpairs, qrow = (u - h * n_qpairs) * kPairRows + prow;
+  if (qrow >= lq) return;
+  const int64_t W = static_cast<int64_t>(n_units) * n_tiles;
+  const int64_t ustart = static_cast<int64_t>(u) * n_tiles, uend = ustart + n_tiles;
+  auto start_of = [&](int c) { return static_cast<int64_t>(c) * W / G; };
+  int c = static_cast<int>(ustart * G / W);
+  if (c >= G) c = G - 1;
+  while (c > 0 && start_of(c) > ustart) --c;
+  while (c + 1 < G && start_of(c + 1) <= ustart) ++c;
+  if (start_of(c) <= ustart && start_of(c + 1) >= uend) return;   // one CTA covered the whole unit
+  int slot[kMaxPieces];
+  int np = 0;
+  for (int cc = c; cc < G && start_of(cc) < uend && np < kMaxPieces; ++cc) {
+    const int64_t sc = start_of(cc), ec = start_of(cc + 1);
+    if (ec <= ustart || ec == sc) continue;
+    const int64_t ps = sc > ustart ? sc : ustart;
+    slot[np++] = 2 * cc + (ps == sc ? 0 : 1);
+  }
   float mx = -INFINITY;
-  for (int s = 0; s < splits; ++s) mx = fmaxf(mx, lsepart[(static_cast<int64_t>(s) * H + h) * lq_pad + qrow]);
+  for (int s = 0; s < np; ++s) mx = fmaxf(mx, lsepart[static_cast<int64_t>(slot[s]) * kPairRows + prow]);
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float wsum = 0.f;
-  for (int s = 0; s < splits; ++s) {
-    const int64_t idx = (static_cast<int64_t>(s) * H + h) * lq_pad + qrow;
+  for (int s = 0; s < np; ++s) {
+    const int64_t idx = static_cast<int64_t>(slot[s]) * kPairRows + prow;
     const float ls = lsepart[idx];
     const float w = (ls == -INFINITY) ? 0.f : expf(ls - mx);
     const float4 o = reinterpret_cast<const float4*>(opart + idx * kHeadDim)[lane];
@@ -418,14 +663,25 @@ combine_kernel(const float* __restrict__ opart, const float* __restrict__ lsepar
 
 }  // namespace
 
+int attention_partial_slots(int n_heads, int max_lq, int max_splits) {
+  const int units = n_heads * ((max_lq + kPairRows - 1) / kPairRows);
+  const int by_split = units * (max_splits > 1 ? max_splits : 1);
+  return 2 * (by_split > 256 ? by_split : 256);
+}
+
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
                            cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kSmemBytes)));
-    attr_set = true;
+  static int npoly = -1;
+  if (npoly < 0) {
+    const char* e = getenv("WK_ATTN_POLY");
+    npoly = e ? atoi(e) : kDefaultPoly;
+    if (npoly < 0 || npoly > 4) npoly = kDefaultPoly;
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
   }
   AttnParams p;
   wk_status st = encode_rows_map(ctx, Q, lq, kTileQ, &p.tm_q);
@@ -462,33 +718,42 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   p.n_tiles = tiles + n_slots * p.tiles_per_slot;
   p.lq = lq;
   p.H = ctx->cfg.n_heads;
-  p.lq_pad = static_cast<int>(align_up(static_cast<size_t>(ctx->max_lq), 2 * kTileQ));
+  p.n_qpairs = (lq + kPairRows - 1) / kPairRows;
+  p.n_units = p.n_qpairs * p.H;
   p.scale_log2 = ctx->scale * 1.4426950408889634f;
   p.O = O;
   p.lse = lse;
   p.opart = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.opart_off);
   p.lsepart = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.lsepart_off);
   p.status = ctx->status_dev;
-  const int n_qpairs = (lq + 2 * kTileQ - 1) / (2 * kTileQ);
-  const int units = n_qpairs * p.H;
-  int splits = kv_splits;
-  const int max_splits = ctx->max_splits > 1 ? ctx->max_splits : 1;
-  if (splits == 0) {
-    // fill the SMs when there are few (head, q-pair) units, but keep at least 8 KV tiles per split
-    splits = ctx->sm_count / units;
-    const int by_tiles = p.n_tiles / 8;
-    if (splits > by_tiles) splits = by_tiles;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
+  const int64_t W = static_cast<int64_t>(p.n_units) * p.n_tiles;
+  int64_t G;
+  if (kv_splits == 0) {
+    G = ctx->sm_count;                       // equal shares of the unit x tile space, one CTA per SM
+    if (G > static_cast<int64_t>(p.n_units) * (kMaxPieces - 2)) G = static_cast<int64_t>(p.n_units) * (kMaxPieces - 2);
+  } else if (kv_splits > 0) {
+    int sp = kv_splits < p.n_tiles ? kv_splits : p.n_tiles;
+    if (sp > kMaxPieces) sp = kMaxPieces;
+    G = static_cast<int64_t>(p.n_units) * sp;  // every unit cut into exactly sp ranges
+  } else {
+    G = -static_cast<int64_t>(kv_splits);      // caller-chosen number of equal ranges
+    if (G * p.n_tiles > W * (kMaxPieces - 2)) return WK_ERR_SHAPE;   // a unit would be cut into too many pieces
   }
-  if (splits > p.n_tiles) splits = p.n_tiles;
-  p.splits = splits;
-  const dim3 grid(n_qpairs, p.H, splits);
-  memory_attention_kernel<<<grid, kThreads, kSmemBytes, s>>>(p);
+  if (G > W) G = W;
+  const int max_slots = attention_partial_slots(p.H, ctx->max_lq, ctx->max_splits);
+  if (2 * G > max_slots) return WK_ERR_SHAPE;
+  switch (npoly) {
+    case 0: memory_attention_kernel<0><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
+    case 1: memory_attention_kernel<1><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
+    case 2: memory_attention_kernel<2><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
+    case 3: memory_attention_kernel<3><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
+    default: memory_attention_kernel<4><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
+  }
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  if (splits > 1) {
-    const int warps = lq * p.H;
-    combine_kernel<<<(warps * 32 + 255) / 256, 256, 0, s>>>(p.opart, p.lsepart, splits, p.H, lq, p.lq_pad, O, lse);
+  if (G != p.n_units) {   // some unit was cut
+    const int64_t warps = static_cast<int64_t>(p.n_units) * kPairRows;
+    combine_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, s>>>(
+        p.opart, p.lsepart, static_cast<int>(G), p.n_units, p.n_tiles, p.n_qpairs, p.H, lq, O, lse);
     if ((st = after_launch(ctx)) != WK_OK) return st;
   }
   return WK_OK;

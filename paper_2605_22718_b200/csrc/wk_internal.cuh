@@ -106,6 +106,9 @@ wk_status encode_rows_map(wk_ctx* ctx, const void* base, int64_t rows, int box_r
 wk_status encode_pool_map(wk_ctx* ctx, const void* base, int64_t rows, int64_t n_mats, int box_rows, CUtensorMap* out);
 const CUtensorMap* cached_rows_map(wk_ctx* ctx, const void* base, int32_t rows, wk_status* st);
 
+// Number of fp32 partial-result slots (256 rows x 128 each) the attention kernel may need.
+int attention_partial_slots(int n_heads, int max_lq, int max_splits);
+
 // Kernel launchers (one per translation unit).
 wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int batch, int32_t* keep_idx,
                           float* scores_out, cudaStream_t s);

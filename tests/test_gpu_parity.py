@@ -190,6 +190,7 @@ def test_memory_attention_cfg0_all_rows():
     (129, [127, 300], 2, 2),       # ragged q tiles and ragged segments
     (300, [], 3, 3),               # pool only
     (257, [40, 128, 129, 5], 1, 1),
+    (600, [2000, 77], 3, 2),       # three q-pairs per head, the last without a second Q tile; 20 KV tiles
 ])
 def test_memory_attention_ragged_shapes(lq, seg_rows, n_slots, H):
     T, n_keep = 40, 23                       # C = 63: less than one KV tile per slot
@@ -212,7 +213,9 @@ def test_memory_attention_ragged_shapes(lq, seg_rows, n_slots, H):
     slot_list = [2, 0, 1][:n_slots]
     slots = torch.tensor(slot_list + [-1], dtype=torch.int32, device="cuda")
     O_ref, L_ref = o.memory_attention(Qb.reshape(lq, H, 128), segs_h, sc.pool, layer, slot_list)
-    for splits in (1, 0, 3):
+    # 0: one range per SM; s > 0: s ranges per (head, q-pair); -g: g equal ranges over the whole space, so that one
+    # CTA runs on from a q-pair without a second Q tile into one with it, and the other way round
+    for splits in (1, 0, 3, -2, -4, -5, -7):
         lse = torch.empty((H, lq), dtype=torch.float32, device="cuda")
         O = kv.memory_attention(layer, Q, segs_d, slots, n_slots, lse_out=lse, kv_splits=splits)
         assert kv.poll_status() == (0, 0)
