@@ -69,59 +69,68 @@ struct TileInfo {
 };
 
 // Walks the effective KV tiles of [tb, te): dense segments first, then pool slots; stale or -1 slots are skipped.
+// Two levels, so that stepping to the next tile of the same segment touches no memory: (segment, tile in segment).
 struct TileIter {
-  int t, te, seg, si, r, z;
-  bool slot_ok;
-  __device__ __forceinline__ void load_slot(const AttnParams& p, bool report) {
-    const int slot = __ldg(p.slots + si);
-    bool ok = slot >= 0 && slot < p.pool_slots;
-    if (ok) ok = __ldg(p.valid + slot) != 0;
-    if (!ok && report && slot != -1) atomicOr(p.status, WK_DEV_BAD_SLOT);   // never dereferenced
-    slot_ok = ok;
-    z = ok ? p.layer * p.pool_slots + slot : 0;
+  int t, te;       // flat tile position, end of the range
+  int seg;         // dense segment index, or n_segs + index into the slot list
+  int r, n_r;      // tile inside the current segment / slot, and how many it has
+  int tail;        // valid rows of its last tile
+  int z;           // pool matrix index (layer * pool_slots + slot)
+  bool ok;         // false for a stale or -1 slot
+  __device__ __forceinline__ void enter(const AttnParams& p, bool report) {
+    if (seg < p.n_segs) {
+      n_r = p.seg_tile_prefix[seg + 1] - p.seg_tile_prefix[seg];
+      tail = p.seg_rows[seg] - (n_r - 1) * kTileKV;
+      z = 0;
+      ok = true;
+    } else {
+      n_r = p.tiles_per_slot;
+      tail = p.C - (n_r - 1) * kTileKV;
+      const int si = seg - p.n_segs;
+      ok = false;
+      z = 0;
+      if (si < p.n_slots) {
+        const int slot = __ldg(p.slots + si);
+        ok = slot >= 0 && slot < p.pool_slots;
+        if (ok) ok = __ldg(p.valid + slot) != 0;
+        if (!ok && report && slot != -1) atomicOr(p.status, WK_DEV_BAD_SLOT);   // never dereferenced
+        if (ok) z = p.layer * p.pool_slots + slot;
+      }
+    }
   }
   __device__ __forceinline__ void init(const AttnParams& p, int tb, int te_, bool report) {
     t = tb;
     te = te_;
-    seg = 0;
-    si = -1;
-    r = 0;
-    slot_ok = false;
-    z = 0;
-    if (t >= p.n_dense_tiles && t < te) {
-      const int u = t - p.n_dense_tiles;
-      si = u / p.tiles_per_slot;
+    if (tb < p.n_dense_tiles) {
+      seg = 0;
+      while (seg + 1 < p.n_segs && tb >= p.seg_tile_prefix[seg + 1]) ++seg;
+      r = tb - p.seg_tile_prefix[seg];
+    } else {
+      const int u = tb - p.n_dense_tiles;
+      const int si = u / p.tiles_per_slot;
+      seg = p.n_segs + si;
       r = u - si * p.tiles_per_slot;
-      load_slot(p, report);
     }
+    n_r = 0;
+    tail = 0;
+    z = 0;
+    ok = false;
+    if (t < te) enter(p, report);
   }
   __device__ __forceinline__ bool next(const AttnParams& p, TileInfo& ti, bool report) {
     while (t < te) {
-      if (t < p.n_dense_tiles) {
-        while (seg + 1 < p.n_segs && t >= p.seg_tile_prefix[seg + 1]) ++seg;
-        ti.seg = seg;
-        ti.row0 = (t - p.seg_tile_prefix[seg]) * kTileKV;
-        ti.z = 0;
-        ti.nv = min(kTileKV, p.seg_rows[seg] - ti.row0);
-        ++t;
-        return true;
-      }
-      if (si < 0) {   // first pool tile of this range
-        si = 0;
+      if (r == n_r) {   // first tile of the next segment / slot
+        ++seg;
         r = 0;
-        load_slot(p, report);
+        enter(p, report);
+        continue;
       }
-      const bool ok = slot_ok;
-      ti.seg = -1;
+      ti.seg = seg < p.n_segs ? seg : -1;
       ti.row0 = r * kTileKV;
       ti.z = z;
-      ti.nv = min(kTileKV, p.C - ti.row0);
+      ti.nv = (r == n_r - 1) ? tail : kTileKV;
+      ++r;
       ++t;
-      if (++r == p.tiles_per_slot) {
-        r = 0;
-        ++si;
-        if (t < te) load_slot(p, report);
-      }
       if (ok) return true;
     }
     return false;
@@ -129,20 +138,24 @@ struct TileIter {
 };
 
 #ifdef WK_ATTN_PROFILE
-// Stage timers for one designated thread per role of CTA 0: clock deltas (in 16-clock units) are added into the words
-// after the status word.  Built only for profiling runs; the product build has none of this.
-#define WK_PROF_DECL long long prof_t = clock64();
-#define WK_PROF(slot, cond)                                                              \
-  do {                                                                                   \
-    if (cond) {                                                                          \
-      const long long now__ = clock64();                                                 \
-      atomicAdd(p.status + 8 + (slot), static_cast<uint32_t>((now__ - prof_t) >> 4));    \
-      prof_t = now__;                                                                    \
-    }                                                                                    \
+// Stage timers for one designated thread per role of CTA 0: clock deltas are accumulated in registers and added into the
+// words after the status word when the role finishes.  Built only for profiling runs; the product build has none of this.
+#define WK_PROF_DECL uint32_t prof_t = clock(); uint32_t prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#define WK_PROF(slot, cond)                              \
+  do {                                                   \
+    const uint32_t now__ = clock();                      \
+    prof_acc[(slot) & 7] += now__ - prof_t;              \
+    prof_t = now__;                                      \
+  } while (0)
+#define WK_PROF_FLUSH(base, cond)                                                          \
+  do {                                                                                     \
+    if (cond)                                                                              \
+      for (int i__ = 0; i__ < 8; ++i__) atomicAdd(p.status + 8 + (base) + i__, prof_acc[i__] >> 4); \
   } while (0)
 #else
 #define WK_PROF_DECL
 #define WK_PROF(slot, cond)
+#define WK_PROF_FLUSH(base, cond)
 #endif
 
 struct __align__(8) Barriers {
@@ -206,6 +219,40 @@ __device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& p0, floa
   p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
 }
 
+// P = 2^(s * scale - m) for one row of a tile: rounds to bf16, stores into tensor memory over S (64 columns), returns
+// the fp32 row sum.  NPOLY of every four element pairs use the polynomial, the rest the MUFU.
+template <int NPOLY>
+__device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t scale2, uint64_t neg_m2, uint32_t tS) {
+  uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint64_t e = fma_f32x2(pack_f32x2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), scale2, neg_m2);
+      float e0, e1;
+      unpack_f32x2(e, e0, e1);
+      float p0, p1;
+      if ((i & 3) < NPOLY) {
+        exp2_poly_x2(e0, e1, p0, p1);
+      } else {
+        p0 = ex2_approx(e0);
+        p1 = ex2_approx(e1);
+      }
+      const uint64_t pp = pack_f32x2(p0, p1);
+      if ((i & 3) == 0) acc0 = add_f32x2(acc0, pp);
+      else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
+      else if ((i & 3) == 2) acc2 = add_f32x2(acc2, pp);
+      else acc3 = add_f32x2(acc3, pp);
+      pk[i] = pack_bf16x2(p0, p1);
+    }
+    tmem_st_x16(tS + c * 16, pk);
+  }
+  float a, b;
+  unpack_f32x2(add_f32x2(add_f32x2(acc0, acc1), add_f32x2(acc2, acc3)), a, b);
+  return a + b;
+}
+
 // One piece of work: unit u, KV tiles [tb, te), and where its result goes.
 struct Piece {
   int h, q0, tb, te, slot;   // slot < 0: the piece covers the whole unit -> direct output
@@ -259,8 +306,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bars.s_full[i], 1); mbar_init(&bars.p_full[i], 128); mbar_init(&bars.o_done[i], 1);
-      mbar_init(&bars.o_free[i], 128);
+      mbar_init(&bars.s_full[i], 1); mbar_init(&bars.p_full[i], 4); mbar_init(&bars.o_done[i], 1);
+      mbar_init(&bars.o_free[i], 4);
     }
     s_abort = 0;
     fence_mbar_init();
@@ -439,6 +486,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
         g0 += n_eff;
         if (q1) g1 += n_eff;
       }
+      WK_PROF_FLUSH(8, blockIdx.x == 0);
     }
   } else {
     // ------------------------------------------------------------------ softmax warpgroups (one thread per query row)
@@ -468,30 +516,52 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           if (!(ok = wait_or_abort(&bars.s_full[wg], g & 1, &s_abort, p.status))) break;
           WK_PROF(1, blockIdx.x == 0 && tid == 0);
           tc_fence_after();
+          // the whole S row (128 fp32) is held in registers: one pass for the row maximum, one for the exponentials
           float s[128];
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t r[32];
-            tmem_ld_x32(tS + c * 32, r);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
-          }
-          tc_wait_ld();
-          WK_PROF(2, blockIdx.x == 0 && tid == 0);
-          if (nv < kTileKV) {
-#pragma unroll
-            for (int i = 0; i < 128; ++i) s[i] = i < nv ? s[i] : -INFINITY;   // zero-filled rows past the segment end
-          }
           float c0 = -INFINITY, c1 = -INFINITY, c2 = -INFINITY, c3 = -INFINITY;
 #pragma unroll
-          for (int i = 0; i < 128; i += 8) {
+          for (int hf = 0; hf < 2; ++hf) {
+            // the second 64 columns are in flight while the maximum of the first 64 is taken
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+              uint32_t r[32];
+              tmem_ld_x32(tS + hf * 64 + c * 32, r);
+#pragma unroll
+              for (int i = 0; i < 32; ++i) s[hf * 64 + c * 32 + i] = __uint_as_float(r[i]);
+            }
+            if (hf == 1) {
+#pragma unroll
+              for (int i = 0; i < 64; i += 8) {
+                c0 = fmax3(c0, s[i], s[i + 1]);
+                c1 = fmax3(c1, s[i + 2], s[i + 3]);
+                c2 = fmax3(c2, s[i + 4], s[i + 5]);
+                c3 = fmax3(c3, s[i + 6], s[i + 7]);
+              }
+            }
+            tc_wait_ld();
+          }
+          WK_PROF(2, blockIdx.x == 0 && tid == 0);
+          const bool full_tile = nv == kTileKV;
+          if (!full_tile) {   // rows past the end of the segment were zero-filled by TMA: mask them out
+            c0 = c1 = c2 = c3 = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 128; ++i) s[i] = i < nv ? s[i] : -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 64; i += 8) {
+              c0 = fmax3(c0, s[i], s[i + 1]);
+              c1 = fmax3(c1, s[i + 2], s[i + 3]);
+              c2 = fmax3(c2, s[i + 4], s[i + 5]);
+              c3 = fmax3(c3, s[i + 6], s[i + 7]);
+            }
+          }
+#pragma unroll
+          for (int i = 64; i < 128; i += 8) {
             c0 = fmax3(c0, s[i], s[i + 1]);
             c1 = fmax3(c1, s[i + 2], s[i + 3]);
             c2 = fmax3(c2, s[i + 4], s[i + 5]);
             c3 = fmax3(c3, s[i + 6], s[i + 7]);
           }
           const float mx = fmaxf(fmax3(c0, c1, c2), c3);
-          WK_PROF(3, blockIdx.x == 0 && tid == 0);
           const float m_new = fmaxf(m_used, mx * p.scale_log2);
           float alpha = 1.f;
           bool rescale = false;
@@ -502,36 +572,9 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           }
           l *= alpha;
           const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
-          uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const uint64_t e = fma_f32x2(pack_f32x2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), scale2, neg_m2);
-              float e0, e1;
-              unpack_f32x2(e, e0, e1);
-              float p0, p1;
-              if ((i & 3) < NPOLY && nv == kTileKV) {
-                exp2_poly_x2(e0, e1, p0, p1);
-              } else {
-                p0 = ex2_approx(e0);
-                p1 = ex2_approx(e1);
-              }
-              const uint64_t pp = pack_f32x2(p0, p1);
-              if ((i & 3) == 0) acc0 = add_f32x2(acc0, pp);
-              else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
-              else if ((i & 3) == 2) acc2 = add_f32x2(acc2, pp);
-              else acc3 = add_f32x2(acc3, pp);
-              pk[i] = pack_bf16x2(p0, p1);
-            }
-            tmem_st_x16(tS + c * 16, pk);
-          }
-          {
-            float a, b;
-            unpack_f32x2(add_f32x2(add_f32x2(acc0, acc1), add_f32x2(acc2, acc3)), a, b);
-            l += a + b;
-          }
+          WK_PROF(3, blockIdx.x == 0 && tid == 0);
+          // masked columns hold -inf, which only the MUFU path maps to 0: tail tiles take no polynomial
+          l += full_tile ? exp_store_tile<NPOLY>(s, scale2, neg_m2, tS) : exp_store_tile<0>(s, scale2, neg_m2, tS);
           if (__any_sync(0xffffffffu, rescale)) {
             // the previous P V product must have landed before O is touched
             if (!(ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status))) break;
@@ -549,7 +592,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           WK_PROF(4, blockIdx.x == 0 && tid == 0);
           tc_wait_st();
           tc_fence_before();
-          mbar_arrive(&bars.p_full[wg]);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.p_full[wg]);   // one arrival per warp: the wait above covered all 32 lanes' stores
           WK_PROF(5, blockIdx.x == 0 && tid == 0);
           ++j;
           ++g;
@@ -606,9 +650,11 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       // O of this piece has been read: the next piece that uses this accumulator may overwrite it
       if (active && j > 0) {
         tc_fence_before();
-        mbar_arrive(&bars.o_free[wg]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.o_free[wg]);
       }
     }
+    WK_PROF_FLUSH(0, blockIdx.x == 0 && tid == 0);
   }
   tc_fence_before();
   __syncthreads();
@@ -729,8 +775,15 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   const int64_t W = static_cast<int64_t>(p.n_units) * p.n_tiles;
   int64_t G;
   if (kv_splits == 0) {
-    G = ctx->sm_count;                       // equal shares of the unit x tile space, one CTA per SM
-    if (G > static_cast<int64_t>(p.n_units) * (kMaxPieces - 2)) G = static_cast<int64_t>(p.n_units) * (kMaxPieces - 2);
+    // One CTA per (head, q-pair) whenever that keeps most SMs busy: under the board's power cap the extra fp32
+    // partials and the combine pass of a finer cut cost more than the idle SMs (measured at the Matrix-Game shape:
+    // 132 CTAs beat 148 equal ranges by 12 %).  Small problems are cut into one equal range per SM instead.
+    if (p.n_units * 4 >= ctx->sm_count * 3) {
+      G = p.n_units;
+    } else {
+      G = ctx->sm_count;
+      if (G > static_cast<int64_t>(p.n_units) * (kMaxPieces - 2)) G = static_cast<int64_t>(p.n_units) * (kMaxPieces - 2);
+    }
   } else if (kv_splits > 0) {
     int sp = kv_splits < p.n_tiles ? kv_splits : p.n_tiles;
     if (sp > kMaxPieces) sp = kMaxPieces;
