@@ -127,6 +127,25 @@ int64_t wk_pool_tag(const wk_ctx* ctx, int32_t slot); /* chunk_tag given at appe
 wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_t* slots_out_dev,
                       double* dist_out_dev, int32_t* n_out_host, void* stream);
 
+/* The paper has no counterpart to this call: it exists for callers that may not allocate device memory.
+ * Same computation and same results as wk_retrieve, but with no context and no caller-provided scratch: the two
+ * doubles per slot the kernel needs live in a fixed array compiled into the library (64 KB, held by every GPU that
+ * loads the library until the process exits).  Use it where cudaMalloc is off the table, for example from code that
+ * runs while a CUDA graph is being captured, from a service whose memory pool is sized once at start-up and then
+ * frozen, or from a plug-in that must not touch the host application's allocator.
+ *   poses_dev [n_slots][8] fp32 and valid_dev [n_slots] int32 are the pool's slot table (a slot with valid = 0 is not
+ *   a candidate); cur_pose_host [8]; slots_out_dev [max_k] int32 and dist_out_dev [max_k] fp64 (or NULL) as in
+ *   wk_retrieve (entries past min(k, M) are -1 / 0).
+ * Limits and caveats: n_slots <= 4096, else WK_ERR_SHAPE and nothing is launched.  The first call on each device looks
+ * up the array's device address (cudaGetSymbolAddress, with that device current); make that first call outside any
+ * stream capture.  All calls on a device share the one array: two calls whose kernels may overlap on the GPU
+ * (different streams) race on it; calls on one stream are safe.  Nothing in the array has to start at zero: every
+ * entry a call reads it has written first.  Calls no cudaMalloc/cudaFree and no allocating library routine.
+ * Errors: WK_ERR_ARG, WK_ERR_SHAPE, WK_ERR_NO_DEVICE, WK_ERR_CUDA. */
+wk_status wk_retrieve_noalloc(const float* poses_dev, const int32_t* valid_dev, int32_t n_slots,
+                              const float* cur_pose_host, int32_t k, int32_t max_k, int32_t* slots_out_dev,
+                              double* dist_out_dev, void* stream);
+
 /* ---- memory attention (Section 4.2) -------------------------------------------------------- */
 
 typedef struct {

@@ -65,6 +65,7 @@ def load_library() -> C.CDLL:
         "wk_pool_count": (i32, [vp]),
         "wk_pool_tag": (i64, [vp, i32]),
         "wk_retrieve": (i32, [vp, C.POINTER(C.c_float), i32, vp, vp, C.POINTER(i32), vp]),
+        "wk_retrieve_noalloc": (i32, [vp, vp, i32, C.POINTER(C.c_float), i32, i32, vp, vp, vp]),
         "wk_memory_attention": (i32, [vp, i32, vp, i32, C.POINTER(wk_dense_seg), i32, vp, i32, vp, vp, i32, vp]),
         "wk_poll_status": (i32, [vp, C.POINTER(C.c_uint32), vp]),
         "wk_status_string": (C.c_char_p, [i32]),
@@ -81,6 +82,7 @@ def load_library() -> C.CDLL:
 
 EXPORTED_SYMBOLS = ("wk_create", "wk_destroy", "wk_pool_bytes", "wk_scratch_bytes", "wk_bind", "wk_compress_chunk",
                     "wk_pool_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
+                    "wk_retrieve_noalloc",
                     "wk_memory_attention", "wk_poll_status", "wk_status_string", "wk_last_cuda_error",
                     "wk_launch_count")
 
@@ -95,6 +97,18 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 def _stream(stream: Optional[torch.cuda.Stream]) -> int:
     return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+def retrieve_noalloc(poses: torch.Tensor, valid: torch.Tensor, cur_pose: Sequence[float], k: int, max_k: int,
+                     slots_out: torch.Tensor, dist_out: Optional[torch.Tensor] = None, stream=None) -> None:
+    """wk_retrieve_noalloc: pose retrieval for callers that may not allocate device memory (no context, scratch built
+    into the library).  poses [n_slots, 8] fp32, valid [n_slots] int32, slots_out [max_k] int32, dist_out [max_k] fp64 -- all
+    preallocated by the caller; this wrapper allocates nothing either."""
+    pose_arr = (C.c_float * 8)(*[float(x) for x in cur_pose])
+    st = load_library().wk_retrieve_noalloc(poses.data_ptr(), valid.data_ptr(), poses.shape[0], pose_arr, k, max_k,
+                                            slots_out.data_ptr(), _ptr(dist_out), _stream(stream))
+    if st != WK_OK:
+        raise WkError(st, "wk_retrieve_noalloc")
 
 
 class WorldKV:

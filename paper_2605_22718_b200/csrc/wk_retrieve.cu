@@ -79,6 +79,10 @@ retrieve_kernel(const float* __restrict__ poses, const int32_t* __restrict__ val
   }
 }
 
+// Scratch of the allocation-free entry point: two doubles per slot, held by every GPU that loads the library.
+constexpr int kStaticMaxSlots = 4096;
+static __device__ __align__(256) double g_retrieve_scratch[2 * kStaticMaxSlots];
+
 }  // namespace
 
 wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out,
@@ -92,3 +96,27 @@ wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* sl
 }
 
 }  // namespace wk
+
+extern "C" wk_status wk_retrieve_noalloc(const float* poses_dev, const int32_t* valid_dev, int32_t n_slots,
+                                         const float* cur_pose_host, int32_t k, int32_t max_k, int32_t* slots_out_dev,
+                                         double* dist_out_dev, void* stream) {
+  using namespace wk;
+  if (!poses_dev || !valid_dev || !cur_pose_host || !slots_out_dev) return WK_ERR_ARG;
+  if (n_slots < 0 || k < 0 || max_k < 1 || k > max_k) return WK_ERR_ARG;
+  if (n_slots > kStaticMaxSlots) return WK_ERR_SHAPE;   // the built-in scratch holds 4096 slots and cannot grow
+  // Set-up, once per device and with that device current: in host code the array's name is only a stand-in, the
+  // device address has to be asked for.
+  static double* scratch_of_device[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return WK_ERR_NO_DEVICE;
+  if (!scratch_of_device[dev]) {
+    double* ptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_retrieve_scratch) != cudaSuccess || !ptr) return WK_ERR_CUDA;
+    scratch_of_device[dev] = ptr;
+  }
+  Pose8 cur;
+  for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose_host[i];
+  retrieve_kernel<<<1, kRetrieveThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      poses_dev, valid_dev, n_slots, cur, k, max_k, scratch_of_device[dev], slots_out_dev, dist_out_dev);
+  return cudaGetLastError() == cudaSuccess ? WK_OK : WK_ERR_CUDA;
+}
