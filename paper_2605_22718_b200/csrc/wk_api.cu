@@ -32,8 +32,9 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   s.m32_off = off;   off += align_up(B * D * sizeof(float), 256);
   s.m64_off = off;   off += align_up(B * D * sizeof(double), 256);
   s.s32_off = off;   off += align_up(B * NA * sizeof(float), 256);
-  s.mnorm_off = off; off += align_up(B * sizeof(double), 256);
+  s.mnorm_off = off; off += align_up(B * 32 * sizeof(double), 256);   // up to 32 shares of |m|^2 per problem
   s.part_off = off;  off += align_up(B * s.anchor_parts * D * sizeof(double), 256);
+  s.inv_off = off;   off += align_up(B * c.tokens_per_frame * sizeof(double), 256);
   s.cnt_off = off;   off += align_up(B * sizeof(uint32_t), 256);
   s.dist_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * 2 * sizeof(double), 256);
   const size_t slots = static_cast<size_t>(attention_partial_slots(c.n_heads, max_lq > 0 ? max_lq : 1, max_splits));

@@ -4,8 +4,9 @@
 // The mean over anchors is pulled inside the dot product: s_j = (k_j . m) / |k_j| with
 // m = (1/T) sum_i a_i / |a_i|, so a chunk is read exactly once (3T*D bf16) instead of T^2 times.
 //
-//   anchor_pass   reads the T anchor rows, accumulates m in fp64 (thread-owned columns, rows staged in
-//                 shared memory), reduces the per-CTA partials in a fixed order -> m64, m32 = fp32(m64), |m|
+//   anchor_norms, anchor_accumulate
+//                 read the T anchor rows (the second time from L2): fp64 row norms, then m in fp64 with thread-owned
+//                 columns; the per-CTA slices are added in a fixed order -> m64, m32 = fp32(m64), |m|
 //   score_pass    reads the (F-1)T non-anchor rows once, fp32 dot with the shared-memory-staged m32 and fp32
 //                 norm, warp-shuffle reductions -> s32
 //   select_pass   per problem: the n_keep-th smallest s32 (radix select) is the threshold; tokens further than
@@ -20,7 +21,9 @@ namespace wk {
 namespace {
 
 constexpr int kAnchorThreads = 256;
-constexpr int kAnchorRows = 8;      // rows staged per iteration (one per warp)
+constexpr int kColSplit = 2;          // column halves per row slice in the fp64 accumulation
+constexpr int kMaxNormParts = 32;     // |m|^2 arrives in up to this many per-CTA shares per problem (D <= 16384)
+constexpr int kMaxAnchorParts = 16;   // slices per problem in the fp64 accumulation (matches the scratch layout)
 constexpr int kScoreThreads = 256;
 constexpr int kScoreRowsPerCta = 64;
 constexpr int kSelectThreads = 1024;
@@ -43,106 +46,116 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// anchor pass.  grid = (parts, batch).  NP = column pairs owned by each thread = ceil(D / 512).
+// anchor pass, two streaming kernels with no block barrier in their loops.
+//   anchor_norms:      one warp per anchor row, fp64 squared norm -> 1/|a_i| (0 for a zero key)
+//   anchor_accumulate: grid = (parts * kColSplit, batch), block = D/(8 kColSplit) threads; a thread owns 8 columns and adds
+//                      a_i[8t..] / |a_i| over the rows of its slice in fp64; the anchor rows come from L2 the second
+//                      time.  The last CTA of a problem adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|.
 // ------------------------------------------------------------------------------------------------
-template <int NP>
 __global__ void __launch_bounds__(kAnchorThreads)
-anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int parts,
-            double* __restrict__ partial, uint32_t* __restrict__ counters, double* __restrict__ m64,
-            float* __restrict__ m32, double* __restrict__ mnorm) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  uint32_t* rows = reinterpret_cast<uint32_t*>(smem);                 // [kAnchorRows][D/2] bf16 pairs
-  __shared__ double inv[kAnchorRows];
-  __shared__ double red[kAnchorThreads / 32];
-  __shared__ uint32_t is_last;
-  const int b = blockIdx.y, part = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride;
-  const int halfD = D >> 1, vecs_per_row = D >> 3;
-
-  double acc0[NP], acc1[NP];
+anchor_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, double* __restrict__ inv_norm) {
+  const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
+  if (r >= T) return;
+  const int vecs = D >> 3;
+  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(r) * D);
+  double n2a = 0.0, n2b = 0.0;
+  for (int v0 = lane; v0 < vecs; v0 += 128) {
+    uint4 q[4];
 #pragma unroll
-  for (int i = 0; i < NP; ++i) acc0[i] = acc1[i] = 0.0;
+    for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
+        n2a = fma(x0, x0, n2a);
+        n2b = fma(x1, x1, n2b);
+      }
+    }
+  }
+  const double n2 = warp_sum(n2a + n2b);
+  if (lane == 0) inv_norm[static_cast<int64_t>(b) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
+}
 
-  const int n_blocks = (T + kAnchorRows - 1) / kAnchorRows;
-  for (int blk = part; blk < n_blocks; blk += parts) {
-    const int r0 = blk * kAnchorRows;
-    const int nr = min(kAnchorRows, T - r0);
-    // stage nr rows (contiguous in global memory)
-    const uint4* src = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(r0) * D);
-    uint4* dst = reinterpret_cast<uint4*>(rows);
-    for (int v = tid; v < nr * vecs_per_row; v += kAnchorThreads) dst[v] = __ldg(src + v);
-    __syncthreads();
-    // one warp per row: squared norm in fp64
-    if (warp < nr) {
-      const uint4* rv = reinterpret_cast<const uint4*>(rows + warp * halfD);
-      double n2 = 0.0;
-      for (int v = lane; v < vecs_per_row; v += 32) {
-        uint4 q = rv[v];
-        uint32_t w[4] = {q.x, q.y, q.z, q.w};
+__global__ void __launch_bounds__(512)
+anchor_accumulate(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int parts,
+                  const double* __restrict__ inv_norm, double* __restrict__ partial) {
+  const int b = blockIdx.y, part = blockIdx.x / kColSplit, csplit = blockIdx.x % kColSplit;
+  const int tid = threadIdx.x, nthreads = blockDim.x;
+  const int vecs = D >> 3;
+  const int vec = csplit * nthreads + tid;   // the 16-byte column group this thread owns
+  const uint4* Kb = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride);
+  const double* inv = inv_norm + static_cast<int64_t>(b) * T;
+  if (vec < vecs) {
+    double acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.0;
+    constexpr int U = 8;   // rows in flight per thread
+    for (int r0 = part; r0 < T; r0 += U * parts) {
+      uint4 q[U];
+      double sc[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int r = r0 + u * parts;
+        q[u] = r < T ? __ldg(Kb + static_cast<int64_t>(r) * vecs + vec) : make_uint4(0, 0, 0, 0);
+        sc[u] = r < T ? __ldg(inv + r) : 0.0;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
-          n2 = fma(x0, x0, n2);
-          n2 = fma(x1, x1, n2);
-        }
-      }
-      n2 = warp_sum(n2);
-      if (lane == 0) inv[warp] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // a zero key has cosine 0 with everything
-    }
-    __syncthreads();
-    // thread-owned column pairs: acc += row * (1/|row|)
-#pragma unroll
-    for (int i = 0; i < NP; ++i) {
-      const int q = tid + i * kAnchorThreads;
-      if (q < halfD) {
-        for (int r = 0; r < nr; ++r) {
-          const uint32_t w = rows[r * halfD + q];
-          const double s = inv[r];
-          acc0[i] = fma(bf16_to_f64(w & 0xFFFFu), s, acc0[i]);
-          acc1[i] = fma(bf16_to_f64(w >> 16), s, acc1[i]);
+          acc[2 * e] = fma(bf16_to_f64(w[e] & 0xFFFFu), sc[u], acc[2 * e]);
+          acc[2 * e + 1] = fma(bf16_to_f64(w[e] >> 16), sc[u], acc[2 * e + 1]);
         }
       }
     }
-    __syncthreads();
-  }
-  double* my = partial + (static_cast<int64_t>(b) * parts + part) * D;
+    double* my = partial + (static_cast<int64_t>(b) * parts + part) * D + 8 * vec;
 #pragma unroll
-  for (int i = 0; i < NP; ++i) {
-    const int q = tid + i * kAnchorThreads;
-    if (q < halfD) {
-      my[2 * q] = acc0[i];
-      my[2 * q + 1] = acc1[i];
-    }
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) is_last = (atomicAdd(&counters[b], 1u) == static_cast<uint32_t>(parts - 1));
-  __syncthreads();
-  if (!is_last) return;
-  __threadfence();
-  // the last CTA of this problem adds the partials in a fixed order
-  const double* pb = partial + static_cast<int64_t>(b) * parts * D;
-  double nn = 0.0;
-  for (int c = tid; c < D; c += kAnchorThreads) {
-    double s = 0.0;
-    for (int p = 0; p < parts; ++p) s += __ldcg(pb + static_cast<int64_t>(p) * D + c);
-    s /= static_cast<double>(T);
-    m64[static_cast<int64_t>(b) * D + c] = s;
-    m32[static_cast<int64_t>(b) * D + c] = static_cast<float>(s);
-    nn = fma(s, s, nn);
-  }
-  nn = warp_sum(nn);
-  if (lane == 0) red[warp] = nn;
-  __syncthreads();
-  if (tid == 0) {
-    double t = 0.0;
-    for (int w = 0; w < kAnchorThreads / 32; ++w) t += red[w];
-    mnorm[b] = sqrt(t);
-    counters[b] = 0;   // ready for the next call
+    for (int e = 0; e < 8; ++e) my[e] = acc[e];
   }
 }
 
-// Fallback for very wide rows (D > 5120): same arithmetic, accumulators in shared memory.
+// Adds the row slices of every problem in a fixed order: m64, m32 = fp32(m64) and this CTA's share of |m|^2.
+// grid = (ceil(D / 512), batch), 256 threads, two columns per thread; all loads are issued before the first addition.
+__global__ void __launch_bounds__(256)
+anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, double* __restrict__ m64, float* __restrict__ m32,
+              double* __restrict__ mnorm2_part) {
+  __shared__ double red2[8];
+  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int c = 2 * (blockIdx.x * 256 + tid);
+  const double* pb = partial + static_cast<int64_t>(b) * parts * D;
+  double nn = 0.0;
+  if (c < D) {
+    double2 v[kMaxAnchorParts];
+#pragma unroll
+    for (int p = 0; p < kMaxAnchorParts; ++p)
+      v[p] = p < parts ? __ldcg(reinterpret_cast<const double2*>(pb + static_cast<int64_t>(p) * D + c)) : make_double2(0.0, 0.0);
+    double t0 = 0.0, t1 = 0.0;
+#pragma unroll
+    for (int p = 0; p < kMaxAnchorParts; ++p) {
+      t0 += v[p].x;
+      t1 += v[p].y;
+    }
+    t0 /= static_cast<double>(T);
+    t1 /= static_cast<double>(T);
+    *reinterpret_cast<double2*>(m64 + static_cast<int64_t>(b) * D + c) = make_double2(t0, t1);
+    *reinterpret_cast<float2*>(m32 + static_cast<int64_t>(b) * D + c) = make_float2(static_cast<float>(t0), static_cast<float>(t1));
+    nn = fma(t0, t0, fma(t1, t1, 0.0));
+  }
+  nn = warp_sum(nn);
+  if (lane == 0) red2[warp] = nn;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+    for (int w = 0; w < 8; ++w) t += red2[w];
+    mnorm2_part[static_cast<int64_t>(b) * kMaxNormParts + blockIdx.x] = t;
+  }
+}
+
+// Fallback for very wide rows (D > 8192): same arithmetic, accumulators in shared memory.
 __global__ void __launch_bounds__(kAnchorThreads)
 anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int parts,
                  double* __restrict__ partial, uint32_t* __restrict__ counters, double* __restrict__ m64,
@@ -201,7 +214,7 @@ anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int
   if (tid == 0) {
     double t = 0.0;
     for (int w = 0; w < kAnchorThreads / 32; ++w) t += red[w];
-    mnorm[b] = sqrt(t);
+    mnorm[static_cast<int64_t>(b) * kMaxNormParts] = t;   // |m|^2, a single share
     counters[b] = 0;
   }
 }
@@ -225,40 +238,51 @@ score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
   const int j0 = blockIdx.x * kScoreRowsPerCta;
   const int j1 = min(NA, j0 + kScoreRowsPerCta);
   const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * D;
-  for (int j = j0 + warp; j < j1; j += kScoreThreads / 32) {
-    const uint4* row = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
-    float dot = 0.f, n2 = 0.f;
+  // two rows per warp at a time, so that twice as many 16-byte loads are in flight
+  constexpr int W = kScoreThreads / 32;
+  for (int j = j0 + warp; j < j1; j += 2 * W) {
+    const int jb = j + W;
+    const bool has_b = jb < j1;
+    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
+    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * D);
+    float dot_a = 0.f, n2_a = 0.f, dot_b = 0.f, n2_b = 0.f;
     for (int v0 = lane; v0 < vecs; v0 += 128) {
-      uint4 q[4];
+      uint4 qa[4], qb[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + 32 * u;
-        q[u] = v < vecs ? __ldg(row + v) : make_uint4(0, 0, 0, 0);
+        qa[u] = v < vecs ? __ldg(row_a + v) : make_uint4(0, 0, 0, 0);
+        qb[u] = v < vecs ? __ldg(row_b + v) : make_uint4(0, 0, 0, 0);
       }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + 32 * u;
         if (v < vecs) {
           const float4 ma = m[2 * v], mb = m[2 * v + 1];
-          float x;
-          x = bf16lo(q[u].x); dot = fmaf(x, ma.x, dot); n2 = fmaf(x, x, n2);
-          x = bf16hi(q[u].x); dot = fmaf(x, ma.y, dot); n2 = fmaf(x, x, n2);
-          x = bf16lo(q[u].y); dot = fmaf(x, ma.z, dot); n2 = fmaf(x, x, n2);
-          x = bf16hi(q[u].y); dot = fmaf(x, ma.w, dot); n2 = fmaf(x, x, n2);
-          x = bf16lo(q[u].z); dot = fmaf(x, mb.x, dot); n2 = fmaf(x, x, n2);
-          x = bf16hi(q[u].z); dot = fmaf(x, mb.y, dot); n2 = fmaf(x, x, n2);
-          x = bf16lo(q[u].w); dot = fmaf(x, mb.z, dot); n2 = fmaf(x, x, n2);
-          x = bf16hi(q[u].w); dot = fmaf(x, mb.w, dot); n2 = fmaf(x, x, n2);
+          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+          const uint32_t wa[4] = {qa[u].x, qa[u].y, qa[u].z, qa[u].w}, wb[4] = {qb[u].x, qb[u].y, qb[u].z, qb[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x;
+            x = bf16lo(wa[e]); dot_a = fmaf(x, mm[2 * e], dot_a); n2_a = fmaf(x, x, n2_a);
+            x = bf16hi(wa[e]); dot_a = fmaf(x, mm[2 * e + 1], dot_a); n2_a = fmaf(x, x, n2_a);
+            x = bf16lo(wb[e]); dot_b = fmaf(x, mm[2 * e], dot_b); n2_b = fmaf(x, x, n2_b);
+            x = bf16hi(wb[e]); dot_b = fmaf(x, mm[2 * e + 1], dot_b); n2_b = fmaf(x, x, n2_b);
+          }
         }
       }
     }
-    dot = warp_sum(dot);
-    n2 = warp_sum(n2);
-    if (lane == 0) {
-      const float s = n2 > 0.f ? __fdiv_rn(dot, __fsqrt_rn(n2)) : 0.f;
-      if (!isfinite(s)) atomicOr(status, WK_DEV_NONFINITE);
-      s32[static_cast<int64_t>(b) * NA + j] = s;
-      if (scores_out) scores_out[static_cast<int64_t>(b) * NA + j] = s;
+    dot_a = warp_sum(dot_a);
+    n2_a = warp_sum(n2_a);
+    dot_b = warp_sum(dot_b);
+    n2_b = warp_sum(n2_b);
+    if (lane < 2 && (lane == 0 || has_b)) {
+      const float dot = lane ? dot_b : dot_a, n2 = lane ? n2_b : n2_a;
+      const int jj = lane ? jb : j;
+      const float sc = n2 > 0.f ? __fdiv_rn(dot, __fsqrt_rn(n2)) : 0.f;
+      if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+      s32[static_cast<int64_t>(b) * NA + jj] = sc;
+      if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
     }
   }
 }
@@ -277,7 +301,7 @@ __device__ __forceinline__ float key_f32(uint32_t k) {
 __global__ void __launch_bounds__(kSelectThreads)
 select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int n_keep,
             const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
-            int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
+            int n_norm_parts, int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem);                       // [NA]
   int32_t* band_idx = reinterpret_cast<int32_t*>(keys + NA);                // [NA]
@@ -286,6 +310,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sel_prefix, sel_rank, n_band, n_below;
   __shared__ uint32_t warp_tot[kSelectThreads / 32];
+  __shared__ double band_red[8][kSelectThreads / 32];
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = T + n_keep;
   int32_t* out = keep_idx + static_cast<int64_t>(b) * C;
@@ -310,15 +335,29 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
       if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFFu], 1u);
     }
     __syncthreads();
-    if (tid == 0) {
-      uint32_t r = sel_rank, c = 0;
-      int bin = 0;
-      for (; bin < 256; ++bin) {
-        if (c + hist[bin] > r) break;
-        c += hist[bin];
+    if (warp == 0) {
+      // find the bin in which the cumulative count passes the wanted rank: 8 bins per lane, then a warp scan
+      uint32_t h[8], tot = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { h[i] = hist[lane * 8 + i]; tot += h[i]; }
+      uint32_t incl = tot;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
       }
-      sel_prefix = prefix | (static_cast<uint32_t>(bin) << shift);
-      sel_rank = r - c;
+      const uint32_t r = sel_rank;
+      uint32_t c = incl - tot;                 // count in the bins of lower lanes
+      if (c <= r && r < incl) {                 // exactly one lane holds the crossing
+        int bin = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (c + h[i] <= r) { c += h[i]; bin = i + 1; }
+          else break;
+        }
+        sel_prefix = prefix | (static_cast<uint32_t>(lane * 8 + bin) << shift);
+        sel_rank = r - c;
+      }
     }
     __syncthreads();
   }
@@ -326,7 +365,9 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
   // fp32 error band.  Per lane: n_l = 8*ceil(D/256) products in a fused chain, then 5 shuffle adds, the rounding of
   // m to fp32, the norm (same chain), one sqrt and one division: |s32 - s| <= (2 n_l + 32) 2^-24 |m|.
   const int n_l = 8 * ((D + 255) / 256);
-  const double eps = (2.0 * n_l + 32.0) * 5.9604644775390625e-08 * mnorm[b] * 1.000001;
+  double mn2 = 0.0;
+  for (int i = 0; i < n_norm_parts; ++i) mn2 += mnorm[static_cast<int64_t>(b) * kMaxNormParts + i];
+  const double eps = (2.0 * n_l + 32.0) * 5.9604644775390625e-08 * sqrt(mn2) * 1.000001;
   const double lo = static_cast<double>(theta) - 2.0 * eps;
   const double hi = static_cast<double>(theta) + 2.0 * eps;
   uint32_t my_below = 0;
@@ -342,26 +383,61 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
   __syncthreads();
   const int nb = static_cast<int>(n_band);
   const int need = n_keep - static_cast<int>(n_below);   // >= 1: the threshold token itself is in the band
-  // exact fp64 scores of the band tokens, one warp per token
+  // exact fp64 scores of the band tokens: the whole CTA works on four tokens at a time (thread = one 16-byte vector
+  // of the row), partial sums meet in shared memory and are added in a fixed order
   const __nv_bfloat16* Nb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * D;
   const double* mb = m64 + static_cast<int64_t>(b) * D;
-  for (int t = warp; t < nb; t += kSelectThreads / 32) {
-    const uint16_t* row = reinterpret_cast<const uint16_t*>(Nb + static_cast<int64_t>(band_idx[t]) * D);
-    double dot = 0.0, n2 = 0.0;
-    for (int c = lane; c < D; c += 32) {
-      const double x = bf16_to_f64(row[c]);
-      dot = fma(x, mb[c], dot);
-      n2 = fma(x, x, n2);
+  const int vecs = D >> 3;
+  for (int t0 = 0; t0 < nb; t0 += 4) {
+    double dot[4] = {0.0, 0.0, 0.0, 0.0}, n2[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int v = tid; v < vecs; v += kSelectThreads) {
+      double mv[8];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double2 d2 = __ldcg(reinterpret_cast<const double2*>(mb + 8 * v) + e);
+        mv[2 * e] = d2.x;
+        mv[2 * e + 1] = d2.y;
+      }
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        q[u] = t0 + u < nb ? __ldg(reinterpret_cast<const uint4*>(Nb + static_cast<int64_t>(band_idx[t0 + u]) * D) + v)
+                           : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
+          dot[u] = fma(x0, mv[2 * e], dot[u]);
+          dot[u] = fma(x1, mv[2 * e + 1], dot[u]);
+          n2[u] = fma(x0, x0, n2[u]);
+          n2[u] = fma(x1, x1, n2[u]);
+        }
+      }
     }
-    dot = warp_sum(dot);
-    n2 = warp_sum(n2);
-    if (lane == 0) {
-      const double s = n2 > 0.0 ? dot / sqrt(n2) : 0.0;
-      if (!isfinite(s)) atomicOr(status, WK_DEV_NONFINITE);
-      band_s[t] = s;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      dot[u] = warp_sum(dot[u]);
+      n2[u] = warp_sum(n2[u]);
+      if (lane == 0) {
+        band_red[2 * u][warp] = dot[u];
+        band_red[2 * u + 1][warp] = n2[u];
+      }
     }
+    __syncthreads();
+    if (tid < 4 && t0 + tid < nb) {
+      double d = 0.0, n = 0.0;
+      for (int w = 0; w < kSelectThreads / 32; ++w) {
+        d += band_red[2 * tid][w];
+        n += band_red[2 * tid + 1][w];
+      }
+      const double sc = n > 0.0 ? d / sqrt(n) : 0.0;
+      if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+      band_s[t0 + tid] = sc;
+    }
+    __syncthreads();
   }
-  __syncthreads();
   // rank the band tokens by (score, index); the `need` lowest are kept
   for (int t = tid; t < nb; t += kSelectThreads) {
     const double s = band_s[t];
@@ -419,26 +495,22 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   const int parts = ctx->sl.anchor_parts;
   const bool need_scores = (n_keep > 0 && n_keep < NA) || scores_out != nullptr;
   wk_status st = WK_OK;
+  int n_norm_parts = 1;
   if (need_scores) {
     const dim3 grid_a(parts, batch);
-    const size_t smem_rows = static_cast<size_t>(kAnchorRows) * D * 2;
-    const int np = (D + 511) / 512;
-#define WK_LAUNCH_ANCHOR(NP)                                                                                         \
-  do {                                                                                                               \
-    if (smem_rows > 48 * 1024)                                                                                       \
-      WK_CUDA_TRY(ctx, cudaFuncSetAttribute(anchor_pass<NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,            \
-                                            static_cast<int>(smem_rows)));                                          \
-    anchor_pass<NP><<<grid_a, kAnchorThreads, smem_rows, s>>>(K, stride, T, D, parts, partial, counters, m64, m32,   \
-                                                              mnorm);                                                \
-  } while (0)
-    if (np <= 1) WK_LAUNCH_ANCHOR(1);
-    else if (np <= 2) WK_LAUNCH_ANCHOR(2);
-    else if (np <= 3) WK_LAUNCH_ANCHOR(3);
-    else if (np <= 4) WK_LAUNCH_ANCHOR(4);
-    else if (np <= 6) WK_LAUNCH_ANCHOR(6);
-    else if (np <= 8) WK_LAUNCH_ANCHOR(8);
-    else if (np <= 10) WK_LAUNCH_ANCHOR(10);
-    else {
+    if (D <= 8192) {
+      n_norm_parts = (D + 511) / 512;
+      double* inv_norm = reinterpret_cast<double*>(sc + ctx->sl.inv_off);
+      const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), batch);
+      anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, D, inv_norm);
+      if ((st = after_launch(ctx)) != WK_OK) return st;
+      const int threads = ((D / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
+      const dim3 grid_acc(parts * kColSplit, batch);
+      anchor_accumulate<<<grid_acc, threads, 0, s>>>(K, stride, T, D, parts, inv_norm, partial);
+      if ((st = after_launch(ctx)) != WK_OK) return st;
+      const dim3 grid_r((D + 511) / 512, batch);
+      anchor_reduce<<<grid_r, 256, 0, s>>>(partial, T, D, parts, m64, m32, mnorm);
+    } else {
       const size_t smem_acc = static_cast<size_t>(D) * sizeof(double);
       if (smem_acc > 200 * 1024) return WK_ERR_SHAPE;
       WK_CUDA_TRY(ctx, cudaFuncSetAttribute(anchor_pass_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -446,7 +518,6 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       anchor_pass_wide<<<grid_a, kAnchorThreads, smem_acc, s>>>(K, stride, T, D, parts, partial, counters, m64, m32,
                                                                 mnorm);
     }
-#undef WK_LAUNCH_ANCHOR
     if ((st = after_launch(ctx)) != WK_OK) return st;
     const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, batch);
     score_pass<<<grid_s, kScoreThreads, static_cast<size_t>(D) * sizeof(float), s>>>(K, stride, T, NA, D, m32, s32,
@@ -458,7 +529,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   if (smem_sel > 48 * 1024)
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(smem_sel)));
-  select_pass<<<batch, kSelectThreads, smem_sel, s>>>(K, stride, T, NA, D, n_keep, s32, m64, mnorm, keep_idx,
+  select_pass<<<batch, kSelectThreads, smem_sel, s>>>(K, stride, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts, keep_idx,
                                                      ctx->status_dev);
   return after_launch(ctx);
 }

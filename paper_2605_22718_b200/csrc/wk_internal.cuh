@@ -24,7 +24,7 @@ struct PoolLayout {
 PoolLayout pool_layout(const wk_config& c);
 
 struct ScratchLayout {
-  size_t m32_off, m64_off, s32_off, mnorm_off, part_off, cnt_off;   // compression
+  size_t m32_off, m64_off, s32_off, mnorm_off, part_off, inv_off, cnt_off;   // compression
   size_t dist_off;                                                  // retrieval
   size_t opart_off, lsepart_off;                                    // split-KV partials
   size_t total;
