@@ -119,10 +119,12 @@ def _source_frames(seed: int, layer: int, g0: int, n_frames: int, T: int) -> np.
 
 
 def key_frames_bf16(seed: int, layer: int, g0: int, n_frames: int, T: int, D: int,
-                    sigma: float) -> np.ndarray:
-    """Keys of frames g0 .. g0+n_frames-1 of one layer: uint16 [n_frames*T, D] (bf16 bits)."""
+                    sigma: float, cols=None) -> np.ndarray:
+    """Keys of frames g0 .. g0+n_frames-1 of one layer: uint16 [n_frames*T, D] (bf16 bits).
+    ``cols`` (an index array) restricts the result to those columns of the D-wide rows."""
     src = _source_frames(seed, layer, g0, n_frames, T)  # [n_frames, T]
-    c = np.arange(D, dtype=np.uint64).reshape(1, 1, D)
+    cidx = np.arange(D, dtype=np.uint64) if cols is None else np.asarray(cols, dtype=np.uint64)
+    c = cidx.reshape(1, 1, -1)
     p = np.arange(T, dtype=np.uint64).reshape(1, T, 1)
     g = (g0 + np.arange(n_frames, dtype=np.uint64)).reshape(n_frames, 1, 1)
     with np.errstate(over="ignore"):
@@ -132,22 +134,31 @@ def key_frames_bf16(seed: int, layer: int, g0: int, n_frames: int, T: int, D: in
     eps = normal_f32(seed, STREAM_K_NOISE + layer, eps_idx)
     scaled = (np.float32(sigma) * eps).astype(np.float32)  # fp32 multiply, rounded
     k = (base + scaled).astype(np.float32)  # fp32 add, rounded
-    return f32_to_bf16_bits(k).reshape(n_frames * T, D)
+    return f32_to_bf16_bits(k).reshape(n_frames * T, len(cidx))
 
 
 def key_chunk_bf16(seed: int, layer: int, chunk: int, T: int, D: int, sigma: float,
-                   F: int = 3) -> np.ndarray:
-    """Keys of chunk ``chunk`` (frames F*chunk .. F*chunk+F-1): uint16 [F*T, D]."""
-    return key_frames_bf16(seed, layer, F * chunk, F, T, D, sigma)
+                   F: int = 3, cols=None) -> np.ndarray:
+    """Keys of chunk ``chunk`` (frames F*chunk .. F*chunk+F-1): uint16 [F*T, D] (or [F*T, len(cols)])."""
+    return key_frames_bf16(seed, layer, F * chunk, F, T, D, sigma, cols=cols)
 
 
-def value_chunk_bf16(seed: int, layer: int, chunk: int, T: int, D: int, F: int = 3) -> np.ndarray:
-    """Values of one chunk, i.i.d. unit normals: uint16 [F*T, D]."""
-    n = F * T * D
-    return normal_bf16(seed, STREAM_V + layer, chunk * n, n).reshape(F * T, D)
+def _normal_rows_bf16(seed: int, stream: int, idx0: int, rows: int, D: int, cols=None) -> np.ndarray:
+    """Row-major [rows, D] block of unit normals starting at element idx0, optionally only some columns."""
+    if cols is None:
+        return normal_bf16(seed, stream, idx0, rows * D).reshape(rows, D)
+    cidx = np.asarray(cols, dtype=np.uint64).reshape(1, -1)
+    r = np.arange(rows, dtype=np.uint64).reshape(-1, 1)
+    with np.errstate(over="ignore"):
+        idx = np.uint64(idx0) + r * np.uint64(D) + cidx
+    return f32_to_bf16_bits(normal_f32(seed, stream, idx))
 
 
-def query_bf16(seed: int, layer: int, step: int, chunk: int, Lq: int, D: int) -> np.ndarray:
-    """Queries of one (layer, denoising step, chunk), i.i.d. unit normals: uint16 [Lq, D]."""
-    n = Lq * D
-    return normal_bf16(seed, STREAM_Q + layer * 64 + step, chunk * n, n).reshape(Lq, D)
+def value_chunk_bf16(seed: int, layer: int, chunk: int, T: int, D: int, F: int = 3, cols=None) -> np.ndarray:
+    """Values of one chunk, i.i.d. unit normals: uint16 [F*T, D] (or [F*T, len(cols)])."""
+    return _normal_rows_bf16(seed, STREAM_V + layer, chunk * F * T * D, F * T, D, cols)
+
+
+def query_bf16(seed: int, layer: int, step: int, chunk: int, Lq: int, D: int, cols=None) -> np.ndarray:
+    """Queries of one (layer, denoising step, chunk), i.i.d. unit normals: uint16 [Lq, D] (or [Lq, len(cols)])."""
+    return _normal_rows_bf16(seed, STREAM_Q + layer * 64 + step, chunk * Lq * D, Lq, D, cols)
