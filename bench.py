@@ -190,6 +190,9 @@ class ChunkStepBench:
         self.step_no = 0
         self.attn_events = []
         self.e2e = e2e
+        # buffer sets: set 0 is the resident one; the end-to-end leg double-buffers Q, the denoising chunk's K/V and O
+        # so that host copies of neighbouring steps overlap with compute
+        self.sets = [(self.Q, self.curK, self.curV, self.O)]
         if e2e:
             self.hQ = torch.empty(self.Q.shape, dtype=bf, pin_memory=True)
             self.hQ.copy_(self.Q)
@@ -198,6 +201,10 @@ class ChunkStepBench:
             self.hcurV = torch.empty(self.curV.shape, dtype=bf, pin_memory=True)
             self.hcurV.copy_(self.curV)
             self.hO = torch.empty(self.O.shape, dtype=bf, pin_memory=True)
+            self.sets.append((torch.empty_like(self.Q), torch.empty_like(self.curK), torch.empty_like(self.curV),
+                              torch.empty_like(self.O)))
+            self.h2d_stream = torch.cuda.Stream(device=self.dev)
+            self.d2h_stream = torch.cuda.Stream(device=self.dev)
         torch.cuda.synchronize(self.dev)
         st, flags = self.kv.poll_status()
         if st != 0:
@@ -209,14 +216,11 @@ class ChunkStepBench:
     def attention_calls_per_step(self) -> int:
         return self.w.n_layers * self.w.denoise_steps
 
-    def step(self, record_attention_events: bool = False, host_io: bool = False):
+    def step(self, record_attention_events: bool = False, buffer_set: int = 0):
         torch, w, kv = self.torch, self.w, self.kv
+        Q, curK, curV, O = self.sets[buffer_set]
         i = self.step_no
         self.step_no += 1
-        if host_io:   # the step's inputs arrive from pinned host memory
-            self.Q.copy_(self.hQ, non_blocking=True)
-            self.curK.copy_(self.hcurK, non_blocking=True)
-            self.curV.copy_(self.hcurV, non_blocking=True)
         pose = self.poses[(w.pool_chunks + i) % len(self.poses)]
         _, n = kv.retrieve(pose, w.k, slots_out=self.slots)
         if record_attention_events:
@@ -224,10 +228,10 @@ class ChunkStepBench:
             e0.record()
         for s in range(w.denoise_steps):
             for l in range(w.n_layers):
-                segs = [(self.curK[l], self.curV[l])]
+                segs = [(curK[l], curV[l])]
                 if w.window_frames > 0:
                     segs.append((self.winK[l], self.winV[l]))
-                kv.memory_attention(l, self.Q[l, s], segs, self.slots, n, O=self.O[l, s], kv_splits=self.kv_splits)
+                kv.memory_attention(l, Q[l, s], segs, self.slots, n, O=O[l, s], kv_splits=self.kv_splits)
         if record_attention_events:
             e1.record()
             self.attn_events.append((e0, e1))
@@ -237,17 +241,63 @@ class ChunkStepBench:
         if kv.pool_count() == w.pool_chunks:
             kv.pool_evict(kv.pool_oldest())
         kv.pool_append(0, w.n_layers, self.evK[j], self.evV[j], self.keep, pose, chunk_tag=w.pool_chunks + i)
-        if host_io:   # and its result goes back
-            self.hO.copy_(self.O, non_blocking=True)
 
-    def time_steps(self, steps: int, host_io: bool):
+    def time_steps(self, steps: int):
+        """K chunk steps with every input already resident in HBM."""
         torch = self.torch
         barrier()
         torch.cuda.synchronize(self.dev)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
-            self.step(record_attention_events=not host_io, host_io=host_io)
+            self.step(record_attention_events=True)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        barrier()
+        return e0.elapsed_time(e1)
+
+    def time_steps_e2e(self, steps: int):
+        """K chunk steps through the public calls with HOST buffers: every step's Q and denoising-chunk K/V are copied
+        from pinned host memory and its O is copied back, inside the timed region.  Copies run on two copy streams and
+        are double-buffered, so step i+1's inputs and step i-1's outputs move while step i computes."""
+        torch = self.torch
+        cs = torch.cuda.current_stream(self.dev)
+        ev_h2d, ev_comp, ev_d2h = [None] * steps, [None] * steps, [None] * steps
+
+        def issue_h2d(i):
+            Q, curK, curV, _ = self.sets[i % 2]
+            with torch.cuda.stream(self.h2d_stream):
+                if i >= 2:
+                    self.h2d_stream.wait_event(ev_comp[i - 2])      # the buffers' previous user has finished
+                Q.copy_(self.hQ, non_blocking=True)
+                curK.copy_(self.hcurK, non_blocking=True)
+                curV.copy_(self.hcurV, non_blocking=True)
+                ev_h2d[i] = torch.cuda.Event()
+                ev_h2d[i].record(self.h2d_stream)
+
+        barrier()
+        torch.cuda.synchronize(self.dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        self.h2d_stream.wait_event(e0)
+        issue_h2d(0)
+        for i in range(steps):
+            if i + 1 < steps:
+                issue_h2d(i + 1)
+            cs.wait_event(ev_h2d[i])
+            if i >= 2:
+                cs.wait_event(ev_d2h[i - 2])                         # O of this buffer set has been read back
+            self.step(buffer_set=i % 2)
+            ev_comp[i] = torch.cuda.Event()
+            ev_comp[i].record(cs)
+            with torch.cuda.stream(self.d2h_stream):
+                self.d2h_stream.wait_event(ev_comp[i])
+                self.hO.copy_(self.sets[i % 2][3], non_blocking=True)
+                ev_d2h[i] = torch.cuda.Event()
+                ev_d2h[i].record(self.d2h_stream)
+        cs.wait_event(ev_d2h[steps - 1])
+        if steps >= 2:
+            cs.wait_event(ev_d2h[steps - 2])
         e1.record()
         torch.cuda.synchronize(self.dev)
         barrier()
@@ -358,7 +408,7 @@ def run_ours(args, w: wi.Workload):
         sampler.start()
     if args.profiler_range:   # lets `ncu --profile-from-start off` see the timed steps only
         torch.cuda.cudart().cudaProfilerStart()
-    ms = bench.time_steps(args.steps, host_io=False)
+    ms = bench.time_steps(args.steps)
     if args.profiler_range:
         torch.cuda.cudart().cudaProfilerStop()
     clocks = sampler.stop() if rank == 0 else None
@@ -370,9 +420,8 @@ def run_ours(args, w: wi.Workload):
         raise RuntimeError(f"device status after the timed region: {st} flags {flags}")
     e2e = None
     if not args.no_e2e:
-        for _ in range(1):
-            bench.step(host_io=True)
-        ms_e2e = max_over_ranks(bench.time_steps(args.steps, host_io=True), dev)
+        bench.time_steps_e2e(2)   # warm the copy path
+        ms_e2e = max_over_ranks(bench.time_steps_e2e(args.steps), dev)
     calls = bench.attention_calls_per_step()
     flops_call = bench.attention_flops_per_call()
     flops_step = flops_call * calls
