@@ -69,6 +69,10 @@ WORKLOADS = {
     "cfg2_small": Workload("cfg2_small", seed=2, n_layers=2, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
                            window_frames=6, n_keep=440, pool_chunks=16, k=8, sigma=0.1, denoise_steps=4,
                            trajectory="actions", rollout_chunks=8),
+    # profiling case: all 30 layers (so compression runs at its real batch of 30 problems) with a 4-chunk pool (1 GB)
+    "cfg2_pool4": Workload("cfg2_pool4", seed=2, n_layers=30, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
+                           window_frames=6, n_keep=440, pool_chunks=4, k=4, sigma=0.1, denoise_steps=4,
+                           trajectory="actions", rollout_chunks=8),
     # LingBot-World-Fast-shaped single layer, k swept over {2, 4, 8, 16}
     "cfg3": Workload("cfg3", seed=3, n_layers=1, n_heads=40, head_dim=128, T=1560, F=3, q_frames=3,
                      window_frames=6, n_keep=780, pool_chunks=80, k=8, sigma=0.05, trajectory="loop",
