@@ -256,6 +256,32 @@ class ChunkStepBench:
         barrier()
         return e0.elapsed_time(e1)
 
+    def side_metrics(self, iters: int = 20):
+        """The bandwidth-bound calls timed on their own (CUDA events, rotating input sets larger than L2):
+        wk_compress_chunk over all layers of a chunk, and wk_retrieve."""
+        torch, w, kv = self.torch, self.w, self.kv
+        out = {}
+        for i in range(4):
+            kv.compress_chunk(self.evK[i % len(self.evK)], keep_idx_out=self.keep)
+        torch.cuda.synchronize(self.dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            kv.compress_chunk(self.evK[i % len(self.evK)], keep_idx_out=self.keep)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        us = e0.elapsed_time(e1) / iters * 1e3
+        nbytes = w.n_layers * w.F * w.T * w.D * 2
+        out["compress"] = {"us_per_call": us, "bytes_per_call": nbytes, "gbs": nbytes / us / 1e3, "problems": w.n_layers}
+        pose = self.poses[w.pool_chunks % len(self.poses)]
+        e0.record()
+        for i in range(iters):
+            kv.retrieve(pose, w.k, slots_out=self.slots)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        out["retrieve"] = {"us_per_call": e0.elapsed_time(e1) / iters * 1e3, "candidates": kv.pool_count()}
+        return out
+
     def time_steps_e2e(self, steps: int):
         """K chunk steps through the public calls with HOST buffers: every step's Q and denoising-chunk K/V are copied
         from pinned host memory and its O is copied back, inside the timed region.  Copies run on two copy streams and
@@ -422,6 +448,9 @@ def run_ours(args, w: wi.Workload):
     if not args.no_e2e:
         bench.time_steps_e2e(2)   # warm the copy path
         ms_e2e = max_over_ranks(bench.time_steps_e2e(args.steps), dev)
+    side = bench.side_metrics()
+    side["compress"]["frac_of_hbm_peak"] = side["compress"]["gbs"] / peaks["hbm_gbs"]
+    side["compress"]["peak_gbs"] = peaks["hbm_gbs"]
     calls = bench.attention_calls_per_step()
     flops_call = bench.attention_flops_per_call()
     flops_step = flops_call * calls
@@ -451,6 +480,7 @@ def run_ours(args, w: wi.Workload):
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "memory_attention_kernel"},
+        "compress": side["compress"], "retrieve": side["retrieve"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
     }
