@@ -16,8 +16,6 @@
 //   * warp roles: warps 0-3 / 4-7 = softmax of Q tile 0 / 1 (one thread per row, online softmax in fp32 in
 //     the exp2 domain, running maximum updated lazily), warp 8 = MMA issue, warp 9 = TMA producer.
 // Every wait is bounded; a wait that runs out sets WK_DEV_TIMEOUT, the CTA drains and frees its tensor memory.
-#include <stdlib.h>
-
 #include "ptx_sm100.cuh"
 #include "wk_internal.cuh"
 
@@ -34,7 +32,6 @@ constexpr int kStages = 2;
 constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + 2 * kStages * kTileBytes;   // align slack + Q0,Q1 + K,V stages
 constexpr float kRescaleThreshold = 8.0f;           // log2 units: P stays <= 2^8 between maximum updates
 constexpr int kPairRows = 2 * kTileQ;
-constexpr int kDefaultPoly = 0;
 constexpr int kMaxPieces = 32;                      // most ranges one unit may be cut into
 
 struct AttnParams {
@@ -200,28 +197,9 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
   return d;
 }
 
-// 2^x for a pair of fp32 values in [-126, 9] on the FMA/ALU pipes instead of the MUFU: x = n + f with n = round(x)
-// (magic-number rounding), 2^f by a cubic on [-0.5, 0.5] (relative error 2e-4, ten times below the bf16 rounding
-// P receives anyway), n added into the exponent field.
-__device__ __forceinline__ void exp2_poly_x2(float x0, float x1, float& p0, float& p1) {
-  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
-  const uint64_t x = pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-  const uint64_t xr = add_f32x2(x, magic);                                   // low mantissa bits hold round(x)
-  const uint64_t n = add_f32x2(xr, neg_magic);
-  const uint64_t f = fma_f32x2(n, pack_f32x2(-1.f, -1.f), x);
-  uint64_t q = fma_f32x2(f, pack_f32x2(0.053027522f, 0.053027522f), pack_f32x2(0.24221395f, 0.24221395f));
-  q = fma_f32x2(q, f, pack_f32x2(0.69357258f, 0.69357258f));
-  q = fma_f32x2(q, f, pack_f32x2(0.99995905f, 0.99995905f));
-  float q0, q1, r0, r1;
-  unpack_f32x2(q, q0, q1);
-  unpack_f32x2(xr, r0, r1);
-  p0 = __uint_as_float(__float_as_uint(q0) + (__float_as_uint(r0) << 23));
-  p1 = __uint_as_float(__float_as_uint(q1) + (__float_as_uint(r1) << 23));
-}
-
 // P = 2^(s * scale - m) for one row of a tile: rounds to bf16, stores into tensor memory over S (64 columns), returns
-// the fp32 row sum.  NPOLY of every four element pairs use the polynomial, the rest the MUFU.
-template <int NPOLY>
+// the fp32 row sum.  Every exponential goes to the MUFU: moving a share of them to a polynomial on the FMA pipe was
+// measured slower here (one softmax warp per SM sub-partition is latency-bound, not MUFU-throughput-bound).
 __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t scale2, uint64_t neg_m2, uint32_t tS) {
   uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
 #pragma unroll
@@ -232,13 +210,7 @@ __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t 
       const uint64_t e = fma_f32x2(pack_f32x2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), scale2, neg_m2);
       float e0, e1;
       unpack_f32x2(e, e0, e1);
-      float p0, p1;
-      if ((i & 3) < NPOLY) {
-        exp2_poly_x2(e0, e1, p0, p1);
-      } else {
-        p0 = ex2_approx(e0);
-        p1 = ex2_approx(e1);
-      }
+      const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
       const uint64_t pp = pack_f32x2(p0, p1);
       if ((i & 3) == 0) acc0 = add_f32x2(acc0, pp);
       else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
@@ -283,8 +255,6 @@ struct PieceWalker {
   }
 };
 
-// NPOLY of every four element pairs take the polynomial exp2, the rest the MUFU.
-template <int NPOLY>
 __global__ void __launch_bounds__(kThreads, 1)
 memory_attention_kernel(const __grid_constant__ AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -573,8 +543,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           l *= alpha;
           const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
           WK_PROF(3, blockIdx.x == 0 && tid == 0);
-          // masked columns hold -inf, which only the MUFU path maps to 0: tail tiles take no polynomial
-          l += full_tile ? exp_store_tile<NPOLY>(s, scale2, neg_m2, tS) : exp_store_tile<0>(s, scale2, neg_m2, tS);
+          l += exp_store_tile(s, scale2, neg_m2, tS);   // masked columns hold -inf and come out as 0
           if (__any_sync(0xffffffffu, rescale)) {
             // the previous P V product must have landed before O is touched
             if (!(ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status))) break;
@@ -718,16 +687,11 @@ int attention_partial_slots(int n_heads, int max_lq, int max_splits) {
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
                            cudaStream_t s) {
-  static int npoly = -1;
-  if (npoly < 0) {
-    const char* e = getenv("WK_ATTN_POLY");
-    npoly = e ? atoi(e) : kDefaultPoly;
-    if (npoly < 0 || npoly > 4) npoly = kDefaultPoly;
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kSmemBytes)));
+  static bool attr_set = false;
+  if (!attr_set) {
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kSmemBytes)));
+    attr_set = true;
   }
   AttnParams p;
   wk_status st = encode_rows_map(ctx, Q, lq, kTileQ, &p.tm_q);
@@ -795,13 +759,7 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   if (G > W) G = W;
   const int max_slots = attention_partial_slots(p.H, ctx->max_lq, ctx->max_splits);
   if (2 * G > max_slots) return WK_ERR_SHAPE;
-  switch (npoly) {
-    case 0: memory_attention_kernel<0><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
-    case 1: memory_attention_kernel<1><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
-    case 2: memory_attention_kernel<2><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
-    case 3: memory_attention_kernel<3><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
-    default: memory_attention_kernel<4><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p); break;
-  }
+  memory_attention_kernel<<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p);
   if ((st = after_launch(ctx)) != WK_OK) return st;
   if (G != p.n_units) {   // some unit was cut
     const int64_t warps = static_cast<int64_t>(p.n_units) * kPairRows;
