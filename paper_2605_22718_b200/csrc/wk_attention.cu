@@ -28,8 +28,8 @@ constexpr int kThreads = 320;
 constexpr int kMmaWarp = 8, kTmaWarp = 9;
 constexpr uint32_t kHalfTileBytes = 128 * 64 * 2;   // one TMA box: 128 rows x 64 bf16 = 16 KB
 constexpr uint32_t kTileBytes = 2 * kHalfTileBytes; // 128 x 128 bf16
-constexpr int kStages = 2;
-constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + 2 * kStages * kTileBytes;   // align slack + Q0,Q1 + K,V stages
+constexpr int kStagesK = 3, kStagesV = 2;           // K is wanted one MMA group earlier than V: it gets the spare 32 KB
+constexpr size_t kSmemBytes = 1024 + 2 * kTileBytes + (kStagesK + kStagesV) * kTileBytes;   // align slack + Q0,Q1 + K,V stages
 constexpr float kRescaleThreshold = 8.0f;           // log2 units: P stays <= 2^8 between maximum updates
 constexpr int kPairRows = 2 * kTileQ;
 constexpr int kMaxPieces = 32;                      // most ranges one unit may be cut into
@@ -157,7 +157,7 @@ struct TileIter {
 
 struct __align__(8) Barriers {
   uint64_t q_full, q_empty;
-  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  uint64_t k_full[kStagesK], k_empty[kStagesK], v_full[kStagesV], v_empty[kStagesV];
   uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
 };
 
@@ -261,7 +261,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;                                   // [2 q tiles][2 halves][128 rows][128 B]
   uint8_t* sK = sQ + 2 * kTileBytes;                    // [stages][2 halves][128][128 B]
-  uint8_t* sV = sK + kStages * kTileBytes;
+  uint8_t* sV = sK + kStagesK * kTileBytes;
   __shared__ Barriers bars;
   __shared__ uint32_t s_tmem;
   __shared__ volatile uint32_t s_abort;
@@ -271,10 +271,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
   if (tid == 0) {
     mbar_init(&bars.q_full, 1);
     mbar_init(&bars.q_empty, 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1);
-      mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1);
-    }
+    for (int s = 0; s < kStagesK; ++s) { mbar_init(&bars.k_full[s], 1); mbar_init(&bars.k_empty[s], 1); }
+    for (int s = 0; s < kStagesV; ++s) { mbar_init(&bars.v_full[s], 1); mbar_init(&bars.v_empty[s], 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bars.s_full[i], 1); mbar_init(&bars.p_full[i], 4); mbar_init(&bars.o_done[i], 1);
       mbar_init(&bars.o_free[i], 4);
@@ -311,17 +309,17 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
         TileInfo ti;
         const int x = pc.h * kHeadDim;
         while (it.next(p, ti, true)) {
-          const int st = jk % kStages;
-          const uint32_t ph = (jk / kStages) & 1;
-          if (!(ok = wait_or_abort(&bars.k_empty[st], ph ^ 1, &s_abort, p.status))) break;
-          mbar_expect_tx(&bars.k_full[st], kTileBytes);
-          uint8_t* dk = sK + st * kTileBytes;
+          const int sk = jk % kStagesK, st = jk % kStagesV;
+          const uint32_t phk = (jk / kStagesK) & 1, ph = (jk / kStagesV) & 1;
+          if (!(ok = wait_or_abort(&bars.k_empty[sk], phk ^ 1, &s_abort, p.status))) break;
+          mbar_expect_tx(&bars.k_full[sk], kTileBytes);
+          uint8_t* dk = sK + sk * kTileBytes;
           if (ti.seg >= 0) {
-            tma_load_2d(dk, &p.tm_kd[ti.seg], &bars.k_full[st], x, ti.row0);
-            tma_load_2d(dk + kHalfTileBytes, &p.tm_kd[ti.seg], &bars.k_full[st], x + 64, ti.row0);
+            tma_load_2d(dk, &p.tm_kd[ti.seg], &bars.k_full[sk], x, ti.row0);
+            tma_load_2d(dk + kHalfTileBytes, &p.tm_kd[ti.seg], &bars.k_full[sk], x + 64, ti.row0);
           } else {
-            tma_load_3d(dk, &p.tm_kpool, &bars.k_full[st], x, ti.row0, ti.z);
-            tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[st], x + 64, ti.row0, ti.z);
+            tma_load_3d(dk, &p.tm_kpool, &bars.k_full[sk], x, ti.row0, ti.z);
+            tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[sk], x + 64, ti.row0, ti.z);
           }
           if (!(ok = wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status))) break;
           mbar_expect_tx(&bars.v_full[st], kTileBytes);
@@ -339,12 +337,12 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       }
       // Do not leave while copies may still be landing in shared memory: wait (bounded) for the loads issued last.
       if (s_abort) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < kStagesK; ++s)
           for (uint32_t i = 0; i < (1u << 16); ++i)
             if (mbar_try_wait(&bars.k_full[s], 0) || mbar_try_wait(&bars.k_full[s], 1)) break;
+        for (int s = 0; s < kStagesV; ++s)
           for (uint32_t i = 0; i < (1u << 16); ++i)
             if (mbar_try_wait(&bars.v_full[s], 0) || mbar_try_wait(&bars.v_full[s], 1)) break;
-        }
       }
     }
   } else if (warp == kMmaWarp) {
@@ -408,8 +406,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           ++e1;
         }
         {
-          const int st = g0 % kStages;
-          if (!(ok = wait_or_abort(&bars.k_full[st], (g0 / kStages) & 1, &s_abort, p.status))) break;
+          const int st = g0 % kStagesK;
+          if (!(ok = wait_or_abort(&bars.k_full[st], (g0 / kStagesK) & 1, &s_abort, p.status))) break;
           tc_fence_after();
           issue_s(0, st);
           mma_commit(&bars.s_full[0]);
@@ -419,8 +417,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
         }
         for (int j = 0; j < n_eff; ++j) {
           const uint32_t g = g0 + j;
-          const int st = g % kStages, stn = (g + 1) % kStages;
-          const uint32_t ph = (g / kStages) & 1, phn = ((g + 1) / kStages) & 1;
+          const int st = g % kStagesV, stn = (g + 1) % kStagesK;   // V stage of this tile, K stage of the next
+          const uint32_t ph = (g / kStagesV) & 1, phn = ((g + 1) / kStagesK) & 1;
           const bool more = j + 1 < n_eff;
           WK_PROF(10, blockIdx.x == 0);
           if (!(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
