@@ -134,7 +134,7 @@ class ChunkStepBench:
         torch.cuda.set_device(self.dev)
         L, H, T, D = w.n_layers, w.n_heads, w.T, w.D
         self.kv = WorldKV(n_layers=L, n_heads=H, tokens_per_frame=T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
-                          max_k=max(w.k, 1), max_dense_segments=2, device=device_index, max_batch=L, max_lq=w.Lq,
+                          max_k=max(w.k, 1), max_dense_segments=1 + w.window_segments, device=device_index, max_batch=L, max_lq=w.Lq,
                           max_splits=8)
         bf = torch.bfloat16
         n_poses = w.pool_chunks + 4096
@@ -230,7 +230,9 @@ class ChunkStepBench:
             for l in range(w.n_layers):
                 segs = [(curK[l], curV[l])]
                 if w.window_frames > 0:
-                    segs.append((self.winK[l], self.winV[l]))
+                    rows = self.winK.shape[1] // w.window_segments
+                    for i in range(w.window_segments):
+                        segs.append((self.winK[l, i * rows:(i + 1) * rows], self.winV[l, i * rows:(i + 1) * rows]))
                 kv.memory_attention(l, Q[l, s], segs, self.slots, n, O=O[l, s], kv_splits=self.kv_splits)
         if record_attention_events:
             e1.record()

@@ -127,6 +127,40 @@ def test_cfg1_matrix_game_single_layer():
     assert float((O2.float() - O.float()).abs().max()) <= 2e-3
 
 
+def test_paper_default_window_matrix_game_shape():
+    """Section 5.1's window: sink 3 + retrieved 9 (six compressed chunks) + recent 3 + denoising 3 = 18 latent frames,
+    passed as three dense segments plus six pool slots."""
+    from paper_2605_22718_b200 import WorldKV
+    w = wi.WORKLOADS["paper_mg"]
+    assert w.Lkv == 18 * w.T
+    kv = WorldKV(n_layers=1, n_heads=w.n_heads, tokens_per_frame=w.T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
+                 max_k=w.k, max_batch=1, max_lq=w.Lq, max_splits=2, max_dense_segments=3)
+    poses = wi.loop_poses(w.seed, w.pool_chunks + 3)
+    keeps = fill_pool_on_device(kv, w, poses)
+    cur_chunk = w.pool_chunks + 2
+    slots, n = kv.retrieve(poses[cur_chunk], w.k)
+    ref_slots, _, margin = o.retrieve(poses[cur_chunk], poses[:w.pool_chunks], list(range(w.pool_chunks)), w.k)
+    assert margin > 1e-9 and n == 6
+    np.testing.assert_array_equal(slots.cpu().numpy()[:n], ref_slots)
+    keep_of = {}
+    for c in ref_slots.tolist():
+        idx, _, m = o.compress_chunk(wi.key_chunk_bf16(w.seed, 0, c, w.T, w.D, w.sigma), w.T, w.n_keep)
+        assert m > 1e-11
+        np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), idx)
+        keep_of[c] = idx
+    Q = torch.empty((w.Lq, w.n_heads, 128), dtype=torch.bfloat16, device="cuda")
+    wd.query(Q, w.seed, 0, 0, cur_chunk)
+    cur = dense_rows_device(w, 0, [cur_chunk], w.Lq)
+    sink = dense_rows_device(w, 0, [w.pool_chunks + 4], 3 * w.T)       # any chunk that is not in the pool
+    recent = dense_rows_device(w, 0, [w.pool_chunks + 1], 3 * w.T)
+    lse = torch.empty((w.n_heads, w.Lq), dtype=torch.float32, device="cuda")
+    O = kv.memory_attention(0, Q, [sink, recent, cur], slots, n, lse_out=lse)
+    assert kv.poll_status() == (0, 0)
+    check_sampled_attention(w, 0, O, lse, (0, cur_chunk),
+                            [([w.pool_chunks + 4], 3 * w.T), ([w.pool_chunks + 1], 3 * w.T), ([cur_chunk], w.Lq)],
+                            ref_slots.tolist(), keep_of, heads=[2, 9], rows=SAMPLE_ROWS[w.Lq])
+
+
 def test_cfg3_lingbot_single_layer_and_k_sweep():
     from paper_2605_22718_b200 import WorldKV
     w = wi.WORKLOADS["cfg3"]

@@ -30,6 +30,7 @@ class Workload:
     trajectory: str = "loop"           # "random" | "loop" | "actions"
     k_sweep: Tuple[int, ...] = field(default_factory=tuple)
     rollout_chunks: int = 0
+    window_segments: int = 1           # the dense window is passed as this many equal segments (e.g. sink + recent)
 
     @property
     def D(self) -> int:
@@ -77,6 +78,14 @@ WORKLOADS = {
     "cfg3": Workload("cfg3", seed=3, n_layers=1, n_heads=40, head_dim=128, T=1560, F=3, q_frames=3,
                      window_frames=6, n_keep=780, pool_chunks=80, k=8, sigma=0.05, trajectory="loop",
                      k_sweep=(2, 4, 8, 16)),
+    # the paper's own window (Section 5.1): 18 latent frames = sink 3 + retrieved 9 (six chunks compressed to 1.5
+    # frames each) + recent 3 + denoising 3, on both model shapes; sink and recent are separate dense segments
+    "paper_mg": Workload("paper_mg", seed=5, n_layers=1, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
+                         window_frames=6, n_keep=440, pool_chunks=125, k=6, sigma=0.1, trajectory="loop",
+                         window_segments=2),
+    "paper_lb": Workload("paper_lb", seed=6, n_layers=1, n_heads=40, head_dim=128, T=1560, F=3, q_frames=3,
+                         window_frames=6, n_keep=780, pool_chunks=80, k=6, sigma=0.05, trajectory="loop",
+                         window_segments=2),
     # full-KV stress: the whole uncompressed one-minute history (125 x 2,640 = 330,000 tokens)
     "cfg4": Workload("cfg4", seed=4, n_layers=1, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
                      window_frames=0, n_keep=1760, pool_chunks=125, k=125, sigma=0.1, trajectory="loop"),
