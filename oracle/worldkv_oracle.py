@@ -276,3 +276,47 @@ def memory_attention(Q, dense_segments, pool: Optional[PoolModel], layer: int, s
     """Attention of one layer's query chunk over the assembled KV set."""
     K, V = assemble_kv(dense_segments, pool, layer, slots)
     return attention(Q, K, V, scale=scale, rows=rows)
+
+
+# --------------------------------------------------------------------------------------
+# Query-based retrieval (Appendix C: rank stored chunks by their attention score with
+# respect to the current denoising query)
+# --------------------------------------------------------------------------------------
+# Reading taken (the paper gives no formula): the score of a stored chunk is the attention mass the
+# current queries put on that chunk's stored keys when they attend over ALL stored chunks of the
+# layer, averaged over heads and query rows; the k largest scores win, ties to the lowest slot.
+
+
+def query_scores(Q, pool: PoolModel, layer: int, scale: Optional[float] = None):
+    """Returns (slots ascending, score per slot).  Scores are non-negative and sum to 1."""
+    slots = pool.valid_slots()
+    Qf = _as_f64(Q)
+    Lq, H, d = Qf.shape
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    if not slots:
+        return slots, np.zeros(0)
+    lse = np.empty((len(slots), H, Lq))
+    for n, s in enumerate(slots):
+        Ks = _as_f64(pool.K[(layer, s)])
+        for h in range(H):
+            S = scale * (Qf[:, h, :] @ Ks[:, h, :].T)               # [Lq, C]
+            mx = S.max(axis=1)
+            lse[n, h] = mx + np.log(np.exp(S - mx[:, None]).sum(axis=1))
+    top = lse.max(axis=0)
+    w = np.exp(lse - top)                                            # [M, H, Lq]
+    mass = w / w.sum(axis=0)                                         # softmax mass of each chunk, per head and row
+    return slots, mass.mean(axis=(1, 2))
+
+
+def retrieve_query(Q, pool: PoolModel, layer: int, k: int, scale: Optional[float] = None):
+    """Top-k chunks by query_scores.  Returns (slot ids in rank order, their scores, margin to rank k+1)."""
+    slots, score = query_scores(Q, pool, layer, scale)
+    slots = np.asarray(slots, dtype=np.int64)
+    order = np.lexsort((slots, -score))
+    kk = min(k, len(slots))
+    chosen = order[:kk]
+    margin = float("inf")
+    if 0 < kk < len(slots):
+        margin = float(score[order[kk - 1]] - score[order[kk]])
+    return slots[chosen].astype(np.int32), score[chosen], margin
