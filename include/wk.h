@@ -127,6 +127,16 @@ int64_t wk_pool_tag(const wk_ctx* ctx, int32_t slot); /* chunk_tag given at appe
 wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_t* slots_out_dev,
                       double* dist_out_dev, int32_t* n_out_host, void* stream);
 
+/* Query-based retrieval (Appendix C: stored chunks ranked "by their attention scores with respect to the current
+ * denoising query"; the paper gives no formula).  Score of a stored chunk = the softmax mass the queries Q put on that
+ * chunk's stored keys of `layer` when they attend over all stored chunks, averaged over heads and query rows (scores
+ * are >= 0 and sum to 1); the min(k, M) largest win, ties to the lowest slot, written in rank order.
+ *   Q [lq][H][128] bf16; slots_out_dev [max_k] int32 (-1 past the count); score_out_dev [max_k] fp32 or NULL.
+ * Cost: one Q K^T pass over every stored chunk of the layer (the P V half of attention is skipped).
+ * Errors: WK_ERR_SHAPE (lq > max_lq, k > max_k, layer out of range, pool_slots > 1024), WK_ERR_ARG, WK_ERR_UNBOUND. */
+wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, int32_t k, int32_t* slots_out_dev,
+                            float* score_out_dev, int32_t* n_out_host, void* stream);
+
 /* The paper has no counterpart to this call: it exists for callers that may not allocate device memory.
  * Same computation and same results as wk_retrieve, but with no context and no caller-provided scratch: the two
  * doubles per slot the kernel needs live in a fixed array compiled into the library (64 KB, held by every GPU that

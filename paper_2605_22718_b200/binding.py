@@ -65,6 +65,7 @@ def load_library() -> C.CDLL:
         "wk_pool_count": (i32, [vp]),
         "wk_pool_tag": (i64, [vp, i32]),
         "wk_retrieve": (i32, [vp, C.POINTER(C.c_float), i32, vp, vp, C.POINTER(i32), vp]),
+        "wk_retrieve_query": (i32, [vp, i32, vp, i32, i32, vp, vp, C.POINTER(i32), vp]),
         "wk_retrieve_noalloc": (i32, [vp, vp, i32, C.POINTER(C.c_float), i32, i32, vp, vp, vp]),
         "wk_memory_attention": (i32, [vp, i32, vp, i32, C.POINTER(wk_dense_seg), i32, vp, i32, vp, vp, i32, vp]),
         "wk_poll_status": (i32, [vp, C.POINTER(C.c_uint32), vp]),
@@ -82,7 +83,7 @@ def load_library() -> C.CDLL:
 
 EXPORTED_SYMBOLS = ("wk_create", "wk_destroy", "wk_pool_bytes", "wk_scratch_bytes", "wk_bind", "wk_compress_chunk",
                     "wk_pool_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
-                    "wk_retrieve_noalloc",
+                    "wk_retrieve_noalloc", "wk_retrieve_query",
                     "wk_memory_attention", "wk_poll_status", "wk_status_string", "wk_last_cuda_error",
                     "wk_launch_count")
 
@@ -210,6 +211,18 @@ class WorldKV:
                                   _stream(stream))
         if st != WK_OK:
             raise WkError(st, "wk_retrieve")
+        return slots_out, n_out.value
+
+    def retrieve_query(self, layer: int, Q: torch.Tensor, k: int, slots_out: Optional[torch.Tensor] = None,
+                       score_out: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, int]:
+        """Query-based retrieval: returns (slots_out int32[max_k] on the device, count = min(k, M))."""
+        if slots_out is None:
+            slots_out = torch.empty(max(1, self.max_k), dtype=torch.int32, device=self.device)
+        n_out = C.c_int32(0)
+        st = self.lib.wk_retrieve_query(self.ctx, layer, Q.data_ptr(), Q.shape[0], k, slots_out.data_ptr(), _ptr(score_out),
+                                        C.byref(n_out), _stream(stream))
+        if st != WK_OK:
+            raise WkError(st, "wk_retrieve_query")
         return slots_out, n_out.value
 
     # ---- memory attention ---------------------------------------------------------------------

@@ -40,6 +40,12 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   const size_t slots = static_cast<size_t>(attention_partial_slots(c.n_heads, max_lq > 0 ? max_lq : 1, max_splits));
   s.opart_off = off;   off += align_up(slots * 2 * kTileQ * kHeadDim * sizeof(float), 256);
   s.lsepart_off = off; off += align_up(slots * 2 * kTileQ * sizeof(float), 256);
+  // query-based retrieval: per-slot log-sum-exp of the query [slot][H][max_lq], identity slot ids, per-block masses
+  const size_t lq1 = static_cast<size_t>(max_lq > 0 ? max_lq : 1);
+  s.qr_blocks = static_cast<int>((static_cast<size_t>(c.n_heads) * lq1 + 255) / 256);
+  s.qr_lse_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * c.n_heads * lq1 * sizeof(float), 256);
+  s.qr_ids_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * sizeof(int32_t), 256);
+  s.qr_part_off = off; off += align_up(static_cast<size_t>(s.qr_blocks) * c.pool_slots * sizeof(double), 256);
   s.total = off;
   return s;
 }
@@ -202,6 +208,12 @@ wk_status wk_bind(wk_ctx* ctx, void* pool_dev, size_t pool_bytes, void* scratch_
   if (st != WK_OK) return st;
   // the anchor pass counts finished CTAs per problem in scratch; the counters must start at zero
   WK_CUDA_TRY(ctx, cudaMemset(ctx->scratch_base + sl.cnt_off, 0, sl.dist_off - sl.cnt_off));
+  {
+    std::vector<int32_t> ids(ctx->cfg.pool_slots);
+    for (int i = 0; i < ctx->cfg.pool_slots; ++i) ids[i] = i;
+    WK_CUDA_TRY(ctx, cudaMemcpy(ctx->scratch_base + sl.qr_ids_off, ids.data(), ids.size() * sizeof(int32_t),
+                                cudaMemcpyHostToDevice));
+  }
   ctx->bound = true;
   return WK_OK;
 }
@@ -303,6 +315,19 @@ wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_
   const int M = wk_pool_count(ctx);
   *n_out_host = k < M ? k : M;
   return launch_retrieve(ctx, cur_pose_host, k, slots_out_dev, dist_out_dev, static_cast<cudaStream_t>(stream));
+}
+
+wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, int32_t k, int32_t* slots_out_dev,
+                            float* score_out_dev, int32_t* n_out_host, void* stream) {
+  if (!ctx || !Q || !slots_out_dev || !n_out_host || lq < 1) return WK_ERR_ARG;
+  if (!ctx->bound) return WK_ERR_UNBOUND;
+  if (!aligned16(Q)) return WK_ERR_ARG;
+  if (layer < 0 || layer >= ctx->cfg.n_layers || lq > ctx->max_lq || k < 0 || k > ctx->cfg.max_k) return WK_ERR_SHAPE;
+  if (ctx->cfg.pool_slots > 1024) return WK_ERR_SHAPE;
+  const int M = wk_pool_count(ctx);
+  *n_out_host = k < M ? k : M;
+  return launch_retrieve_query(ctx, layer, static_cast<const __nv_bfloat16*>(Q), lq, k, slots_out_dev, score_out_dev,
+                               static_cast<cudaStream_t>(stream));
 }
 
 wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, const wk_dense_seg* segs_host,

@@ -46,6 +46,7 @@ struct AttnParams {
   int n_slots, pool_slots, layer, C, tiles_per_slot;
   int n_tiles, n_qpairs, n_units;
   int lq, H;
+  int lse_only;     // 1: only the log-sum-exp is wanted (query-based retrieval): no P V product, no O
   float scale_log2;
   __nv_bfloat16* O;
   float* lse;
@@ -426,7 +427,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           if (!(ok = wait_or_abort(&bars.p_full[0], g & 1, &s_abort, p.status))) break;
           WK_PROF(12, blockIdx.x == 0);
           tc_fence_after();
-          issue_pv(0, st, j > 0);
+          if (!p.lse_only) issue_pv(0, st, j > 0);
           mma_commit(&bars.o_done[0]);
           if (more) {
             WK_PROF(13, blockIdx.x == 0);
@@ -441,7 +442,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             if (!(ok = wait_or_abort(&bars.p_full[1], (g1 + j) & 1, &s_abort, p.status))) break;
             WK_PROF(16, blockIdx.x == 0);
             tc_fence_after();
-            issue_pv(1, st, j > 0);
+            if (!p.lse_only) issue_pv(1, st, j > 0);
             mma_commit(&bars.o_done[1]);
           }
           mma_commit(&bars.v_empty[st]);
@@ -583,7 +584,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = 0u;
             }
-            if (qrow < p.lq) {
+            if (qrow < p.lq && !p.lse_only) {
               if (pc.slot < 0) {
                 uint4* dst = reinterpret_cast<uint4*>(p.O + (static_cast<int64_t>(qrow) * p.H + pc.h) * kHeadDim + c * 32);
 #pragma unroll
@@ -684,7 +685,7 @@ int attention_partial_slots(int n_heads, int max_lq, int max_splits) {
 
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
-                           cudaStream_t s) {
+                           cudaStream_t s, bool lse_only) {
   static bool attr_set = false;
   if (!attr_set) {
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -725,6 +726,7 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   p.tiles_per_slot = (ctx->C + kTileKV - 1) / kTileKV;
   p.n_tiles = tiles + n_slots * p.tiles_per_slot;
   p.lq = lq;
+  p.lse_only = lse_only ? 1 : 0;
   p.H = ctx->cfg.n_heads;
   p.n_qpairs = (lq + kPairRows - 1) / kPairRows;
   p.n_units = p.n_qpairs * p.H;

@@ -27,6 +27,8 @@ struct ScratchLayout {
   size_t m32_off, m64_off, s32_off, mnorm_off, part_off, inv_off, cnt_off;   // compression
   size_t dist_off;                                                  // retrieval
   size_t opart_off, lsepart_off;                                    // split-KV partials
+  size_t qr_lse_off, qr_ids_off, qr_part_off;                       // query-based retrieval
+  int qr_blocks;
   size_t total;
   int anchor_parts;  // partial-sum slices per problem written by the anchor pass
 };
@@ -118,6 +120,8 @@ wk_status launch_slot_mark(wk_ctx* ctx, int slot, int valid, const float* pose, 
 wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out, cudaStream_t s);
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
-                           cudaStream_t s);
+                           cudaStream_t s, bool lse_only = false);
+wk_status launch_retrieve_query(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, int k, int32_t* slots_out,
+                                float* score_out, cudaStream_t s);
 
 }  // namespace wk

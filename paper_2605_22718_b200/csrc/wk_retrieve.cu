@@ -79,6 +79,74 @@ retrieve_kernel(const float* __restrict__ poses, const int32_t* __restrict__ val
   }
 }
 
+// ---- query-based retrieval (Appendix C) --------------------------------------------------------------------------
+// lse[slot][h][r] holds, for every valid slot, the log-sum-exp of query row r of head h over that slot's stored keys.
+// The softmax mass of a slot for (h, r) is exp(lse[slot] - logsumexp over slots); a slot's score is the mean mass.
+// query_mass: one thread per (h, r); the masses are added over the warp by shuffles, over the block in a fixed order,
+// and every block leaves one partial per slot -- no floating-point atomics, so the ranking is reproducible.
+constexpr int kMassThreads = 256;
+
+__global__ void __launch_bounds__(kMassThreads)
+query_mass(const float* __restrict__ lse, const int32_t* __restrict__ valid, int n_slots, int n_hr,
+           double* __restrict__ block_part /*[gridDim.x][n_slots]*/) {
+  extern __shared__ float warp_part[];   // [8 warps][n_slots]
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int i = blockIdx.x * kMassThreads + tid;
+  const bool live = i < n_hr;
+  float mx = -INFINITY;
+  for (int s = 0; s < n_slots; ++s)
+    if (valid[s] && live) mx = fmaxf(mx, lse[static_cast<int64_t>(s) * n_hr + i]);
+  float den = 0.f;
+  for (int s = 0; s < n_slots; ++s)
+    if (valid[s] && live) den += expf(lse[static_cast<int64_t>(s) * n_hr + i] - mx);
+  const float inv = (live && den > 0.f) ? 1.f / den : 0.f;
+  for (int s = 0; s < n_slots; ++s) {
+    float m = 0.f;
+    if (valid[s] && live) m = expf(lse[static_cast<int64_t>(s) * n_hr + i] - mx) * inv;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m += __shfl_xor_sync(0xffffffffu, m, o);
+    if (lane == 0) warp_part[warp * n_slots + s] = m;
+  }
+  __syncthreads();
+  for (int s = tid; s < n_slots; s += kMassThreads) {
+    double t = 0.0;
+    for (int w = 0; w < kMassThreads / 32; ++w) t += static_cast<double>(warp_part[w * n_slots + s]);
+    block_part[static_cast<int64_t>(blockIdx.x) * n_slots + s] = t;
+  }
+}
+
+// One CTA: adds the blocks' partials in order, ranks the valid slots by (score descending, slot ascending).
+__global__ void __launch_bounds__(1024)
+query_topk(const double* __restrict__ block_part, int n_blocks, const int32_t* __restrict__ valid, int n_slots, int n_hr,
+           int k, int max_k, int32_t* __restrict__ slots_out, float* __restrict__ score_out) {
+  __shared__ double score[1024];
+  const int tid = threadIdx.x;
+  for (int s = tid; s < n_slots; s += 1024) {
+    double t = 0.0;
+    for (int b = 0; b < n_blocks; ++b) t += block_part[static_cast<int64_t>(b) * n_slots + s];
+    score[s] = valid[s] ? t / static_cast<double>(n_hr) : -1.0;   // negative marks "not a candidate"
+  }
+  for (int i = tid; i < max_k; i += 1024) {
+    slots_out[i] = -1;
+    if (score_out) score_out[i] = 0.f;
+  }
+  __syncthreads();
+  for (int s = tid; s < n_slots; s += 1024) {
+    const double v = score[s];
+    if (v < 0.0) continue;
+    int rank = 0;
+    for (int u = 0; u < n_slots; ++u) {
+      const double w = score[u];
+      if (w < 0.0) continue;
+      rank += (w > v) || (w == v && u < s);
+    }
+    if (rank < k) {
+      slots_out[rank] = s;
+      if (score_out) score_out[rank] = static_cast<float>(v);
+    }
+  }
+}
+
 // Scratch of the allocation-free entry point: two doubles per slot, held by every GPU that loads the library.
 constexpr int kStaticMaxSlots = 4096;
 static __device__ __align__(256) double g_retrieve_scratch[2 * kStaticMaxSlots];
@@ -92,6 +160,28 @@ wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* sl
   double* dist = reinterpret_cast<double*>(ctx->scratch_base + ctx->sl.dist_off);
   retrieve_kernel<<<1, kRetrieveThreads, 0, s>>>(ctx->poses_dev, ctx->valid_dev, ctx->cfg.pool_slots, cur, k,
                                                  ctx->cfg.max_k, dist, slots_out, dist_out);
+  return after_launch(ctx);
+}
+
+wk_status launch_retrieve_query(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, int k, int32_t* slots_out,
+                                float* score_out, cudaStream_t s) {
+  const int H = ctx->cfg.n_heads, S = ctx->cfg.pool_slots, n_hr = H * lq;
+  float* lse = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.qr_lse_off);
+  const int32_t* ids = reinterpret_cast<const int32_t*>(ctx->scratch_base + ctx->sl.qr_ids_off);
+  double* part = reinterpret_cast<double*>(ctx->scratch_base + ctx->sl.qr_part_off);
+  wk_status st;
+  // log-sum-exp of the query over each stored chunk alone: the attention kernel in its LSE-only mode, one slot a call
+  for (int slot = 0; slot < S; ++slot) {
+    if (ctx->slots[slot].state != SLOT_VALID) continue;
+    st = launch_attention(ctx, layer, Q, lq, nullptr, 0, ids + slot, 1, nullptr, lse + static_cast<int64_t>(slot) * n_hr, 1, s,
+                          true);
+    if (st != WK_OK) return st;
+  }
+  const int blocks = (n_hr + kMassThreads - 1) / kMassThreads;
+  query_mass<<<blocks, kMassThreads, static_cast<size_t>(kMassThreads / 32) * S * sizeof(float), s>>>(lse, ctx->valid_dev, S,
+                                                                                                     n_hr, part);
+  if ((st = after_launch(ctx)) != WK_OK) return st;
+  query_topk<<<1, 1024, 0, s>>>(part, blocks, ctx->valid_dev, S, n_hr, k, ctx->cfg.max_k, slots_out, score_out);
   return after_launch(ctx);
 }
 
