@@ -46,7 +46,9 @@ struct AttnParams {
   int n_slots, pool_slots, layer, C, tiles_per_slot;
   int n_tiles, n_qpairs, n_units;
   int lq, H;
-  int lse_only;     // 1: only the log-sum-exp is wanted (query-based retrieval): no P V product, no O
+  int lse_only;     // 1: only the log-sum-exp is wanted (query-based retrieval): no V loads, no P V product, no O
+  int slot_units;   // 1: every listed slot is a problem of its own: unit = (slot ordinal, head, q-pair), n_tiles =
+                    //    tiles_per_slot, lse laid out [slot ordinal][H][lq]; stale slots give -inf and are not reported
   float scale_log2;
   __nv_bfloat16* O;
   float* lse;
@@ -229,6 +231,7 @@ __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t 
 // One piece of work: unit u, KV tiles [tb, te), and where its result goes.
 struct Piece {
   int h, q0, tb, te, slot;   // slot < 0: the piece covers the whole unit -> direct output
+  int ord;                   // slot ordinal the unit belongs to (0 unless every slot is its own problem)
   bool has_q1;
 };
 struct PieceWalker {
@@ -242,16 +245,24 @@ struct PieceWalker {
   }
   __device__ __forceinline__ bool next(const AttnParams& p, Piece& pc) {
     if (pos >= end) return false;
-    const int u = static_cast<int>(pos / p.n_tiles);
+    int u = static_cast<int>(pos / p.n_tiles);
     pc.tb = static_cast<int>(pos - static_cast<int64_t>(u) * p.n_tiles);
     const int64_t room = end - pos;
     pc.te = static_cast<int>(min(static_cast<int64_t>(p.n_tiles), pc.tb + room));
-    pc.h = u / p.n_qpairs;
-    pc.q0 = (u - pc.h * p.n_qpairs) * kPairRows;
-    pc.has_q1 = pc.q0 + kTileQ < p.lq;
     const bool full = pc.tb == 0 && pc.te == p.n_tiles;
     pc.slot = full ? -1 : 2 * cta + (pos == start ? 0 : 1);
     pos += pc.te - pc.tb;
+    pc.ord = 0;
+    if (p.slot_units) {   // the unit's tiles are those of one slot: shift the range into that slot's part of the tile space
+      const int base = p.H * p.n_qpairs;
+      pc.ord = u / base;
+      u -= pc.ord * base;
+      pc.tb += pc.ord * p.tiles_per_slot;
+      pc.te += pc.ord * p.tiles_per_slot;
+    }
+    pc.h = u / p.n_qpairs;
+    pc.q0 = (u - pc.h * p.n_qpairs) * kPairRows;
+    pc.has_q1 = pc.q0 + kTileQ < p.lq;
     return true;
   }
 };
@@ -306,10 +317,11 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             tma_load_2d(sQ + i * kTileBytes + half * kHalfTileBytes, &p.tm_q, &bars.q_full, pc.h * kHeadDim + half * 64,
                         pc.q0 + i * kTileQ);
         TileIter it;
-        it.init(p, pc.tb, pc.te, true);
+        const bool report = !p.slot_units;
+        it.init(p, pc.tb, pc.te, report);
         TileInfo ti;
         const int x = pc.h * kHeadDim;
-        while (it.next(p, ti, true)) {
+        while (it.next(p, ti, report)) {
           const int sk = jk % kStagesK, st = jk % kStagesV;
           const uint32_t phk = (jk / kStagesK) & 1, ph = (jk / kStagesV) & 1;
           if (!(ok = wait_or_abort(&bars.k_empty[sk], phk ^ 1, &s_abort, p.status))) break;
@@ -322,6 +334,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             tma_load_3d(dk, &p.tm_kpool, &bars.k_full[sk], x, ti.row0, ti.z);
             tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[sk], x + 64, ti.row0, ti.z);
           }
+          if (p.lse_only) { ++jk; continue; }   // no P V product: V is not fetched
           if (!(ok = wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status))) break;
           mbar_expect_tx(&bars.v_full[st], kTileBytes);
           uint8_t* dv = sV + st * kTileBytes;
@@ -422,7 +435,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           const uint32_t ph = (g / kStagesV) & 1, phn = ((g + 1) / kStagesK) & 1;
           const bool more = j + 1 < n_eff;
           WK_PROF(10, blockIdx.x == 0);
-          if (!(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
+          if (!p.lse_only && !(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
           WK_PROF(11, blockIdx.x == 0);
           if (!(ok = wait_or_abort(&bars.p_full[0], g & 1, &s_abort, p.status))) break;
           WK_PROF(12, blockIdx.x == 0);
@@ -445,7 +458,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             if (!p.lse_only) issue_pv(1, st, j > 0);
             mma_commit(&bars.o_done[1]);
           }
-          mma_commit(&bars.v_empty[st]);
+          if (!p.lse_only) mma_commit(&bars.v_empty[st]);
           if (more) {
             if (q1) { issue_s(1, stn); mma_commit(&bars.s_full[1]); }
             mma_commit(&bars.k_empty[stn]);
@@ -608,7 +621,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           }
           if (qrow < p.lq) {
             if (pc.slot < 0) {
-              if (p.lse) p.lse[static_cast<int64_t>(pc.h) * p.lq + qrow] = lse;
+              if (p.lse) p.lse[(static_cast<int64_t>(pc.ord) * p.H + pc.h) * p.lq + qrow] = lse;
             } else {
               p.lsepart[static_cast<int64_t>(pc.slot) * kPairRows + prow] = lse;
             }
@@ -727,6 +740,7 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   p.n_tiles = tiles + n_slots * p.tiles_per_slot;
   p.lq = lq;
   p.lse_only = lse_only ? 1 : 0;
+  p.slot_units = p.lse_only;
   p.H = ctx->cfg.n_heads;
   p.n_qpairs = (lq + kPairRows - 1) / kPairRows;
   p.n_units = p.n_qpairs * p.H;
@@ -736,9 +750,22 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   p.opart = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.opart_off);
   p.lsepart = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.lsepart_off);
   p.status = ctx->status_dev;
+  if (lse_only) {
+    // every listed slot is scored on its own: one unit per (slot, head, q-pair), each over that slot's tiles only
+    if (n_segs != 0 || n_slots < 1) return WK_ERR_ARG;
+    p.n_tiles = p.tiles_per_slot;
+    p.n_units *= n_slots;
+  }
   const int64_t W = static_cast<int64_t>(p.n_units) * p.n_tiles;
   int64_t G;
-  if (kv_splits == 0) {
+  if (lse_only) {
+    // whole units per CTA (nothing to merge): the largest divisor of the unit count that fits the SMs, unless that
+    // would leave more than a quarter of them idle -- then one CTA per unit
+    G = 1;
+    for (int g = ctx->sm_count < p.n_units ? ctx->sm_count : p.n_units; g >= 1; --g)
+      if (p.n_units % g == 0) { G = g; break; }
+    if (G * 4 < static_cast<int64_t>(ctx->sm_count) * 3 && p.n_units > G) G = p.n_units;
+  } else if (kv_splits == 0) {
     // One CTA per (head, q-pair) whenever that keeps most SMs busy: under the board's power cap the extra fp32
     // partials and the combine pass of a finer cut cost more than the idle SMs (measured at the Matrix-Game shape:
     // 132 CTAs beat 148 equal ranges by 12 %).  Small problems are cut into one equal range per SM instead.
@@ -758,10 +785,10 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   }
   if (G > W) G = W;
   const int max_slots = attention_partial_slots(p.H, ctx->max_lq, ctx->max_splits);
-  if (2 * G > max_slots) return WK_ERR_SHAPE;
+  if (!lse_only && 2 * G > max_slots) return WK_ERR_SHAPE;
   memory_attention_kernel<<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p);
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  if (G != p.n_units) {   // some unit was cut
+  if (!lse_only && G != p.n_units) {   // some unit was cut
     const int64_t warps = static_cast<int64_t>(p.n_units) * kPairRows;
     combine_kernel<<<static_cast<unsigned>((warps * 32 + 255) / 256), 256, 0, s>>>(
         p.opart, p.lsepart, static_cast<int>(G), p.n_units, p.n_tiles, p.n_qpairs, p.H, lq, O, lse);

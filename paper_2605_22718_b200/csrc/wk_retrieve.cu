@@ -169,14 +169,10 @@ wk_status launch_retrieve_query(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, 
   float* lse = reinterpret_cast<float*>(ctx->scratch_base + ctx->sl.qr_lse_off);
   const int32_t* ids = reinterpret_cast<const int32_t*>(ctx->scratch_base + ctx->sl.qr_ids_off);
   double* part = reinterpret_cast<double*>(ctx->scratch_base + ctx->sl.qr_part_off);
-  wk_status st;
-  // log-sum-exp of the query over each stored chunk alone: the attention kernel in its LSE-only mode, one slot a call
-  for (int slot = 0; slot < S; ++slot) {
-    if (ctx->slots[slot].state != SLOT_VALID) continue;
-    st = launch_attention(ctx, layer, Q, lq, nullptr, 0, ids + slot, 1, nullptr, lse + static_cast<int64_t>(slot) * n_hr, 1, s,
-                          true);
-    if (st != WK_OK) return st;
-  }
+  // log-sum-exp of the query over each stored chunk alone: the attention kernel in its LSE-only mode, every pool slot a
+  // problem of its own in one launch (slots that hold nothing come back as -inf and are masked by the valid flags)
+  wk_status st = launch_attention(ctx, layer, Q, lq, nullptr, 0, ids, S, nullptr, lse, 1, s, true);
+  if (st != WK_OK) return st;
   const int blocks = (n_hr + kMassThreads - 1) / kMassThreads;
   query_mass<<<blocks, kMassThreads, static_cast<size_t>(kMassThreads / 32) * S * sizeof(float), s>>>(lse, ctx->valid_dev, S,
                                                                                                      n_hr, part);
