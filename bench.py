@@ -282,6 +282,19 @@ class ChunkStepBench:
         e1.record()
         torch.cuda.synchronize(self.dev)
         out["retrieve"] = {"us_per_call": e0.elapsed_time(e1) / iters * 1e3, "candidates": kv.pool_count()}
+        # query-based retrieval (the appendix variant): the denoising chunk's queries scored against every stored chunk
+        # of one layer; the layer rotates so that successive calls read different pool memory
+        n = max(2, iters // 4)
+        kv.retrieve_query(0, self.Q[0, 0], w.k, slots_out=self.slots)
+        torch.cuda.synchronize(self.dev)
+        e0.record()
+        for i in range(n):
+            kv.retrieve_query((i + 1) % w.n_layers, self.Q[(i + 1) % w.n_layers, 0], w.k, slots_out=self.slots)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        us = e0.elapsed_time(e1) / n * 1e3
+        flops = 2.0 * w.Lq * kv.pool_count() * (w.T + w.n_keep) * w.D
+        out["retrieve_query"] = {"us_per_call": us, "candidates": kv.pool_count(), "tflops": flops / us / 1e6}
         return out
 
     def time_steps_e2e(self, steps: int):
@@ -482,7 +495,7 @@ def run_ours(args, w: wi.Workload):
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "memory_attention_kernel"},
-        "compress": side["compress"], "retrieve": side["retrieve"],
+        "compress": side["compress"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
     }
