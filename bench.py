@@ -32,8 +32,9 @@ METRIC = "memory-attn TFLOP/s over the whole chunk step (attention + retrieval +
 UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per memory_attention_kernel launch from the ncu capture summarised in
-# profiles/ (cfg2 shape, one layer call); None until a capture has been taken for the current kernel.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# profiles/memory_attention_cfg2_shape.md (cfg2 per-call shape: 122.7 MB read + 5.5 MB written); it does not depend on
+# the pool size, so the small-pool capture stands for the full workload.  Other workloads report null.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 128.2e6
 
 
 def load_peaks():
@@ -494,7 +495,8 @@ def run_ours(args, w: wi.Workload):
                       "tflops": achieved, "share_of_step": statistics.mean(attn_ms) / ms_per_step},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "kernel": "memory_attention_kernel"},
+                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if w.name.startswith("cfg2") else None,
+                     "kernel": "memory_attention_kernel"},
         "compress": side["compress"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
