@@ -296,6 +296,29 @@ class ChunkStepBench:
         us = e0.elapsed_time(e1) / n * 1e3
         flops = 2.0 * w.Lq * kv.pool_count() * (w.T + w.n_keep) * w.D
         out["retrieve_query"] = {"us_per_call": us, "candidates": kv.pool_count(), "tflops": flops / us / 1e6}
+        # pose retrieval as a streaming scan over far more candidates than a pool holds (32 bytes per candidate): the
+        # sizes at which "GB/s of retrieval" means something.  Seeded device-side draws: t ~ N(0, I), q = normalised N(0, I4).
+        scan = {}
+        gen = torch.Generator(device=self.dev)
+        gen.manual_seed(1000 + w.seed)
+        ids = torch.empty(16, dtype=torch.int32, device=self.dev)
+        for log2n in (16, 20, 24):
+            n_c = 1 << log2n
+            P = torch.randn((n_c, 8), generator=gen, device=self.dev, dtype=torch.float32)
+            P[:, 4:8] /= P[:, 4:8].norm(dim=1, keepdim=True)
+            P[:, 3] = 0
+            for i in range(3):
+                kv.retrieve_scan(P, pose, 16, ids_out=ids)
+            torch.cuda.synchronize(self.dev)
+            e0.record()
+            for i in range(10):
+                kv.retrieve_scan(P, pose, 16, ids_out=ids)
+            e1.record()
+            torch.cuda.synchronize(self.dev)
+            us = e0.elapsed_time(e1) / 10 * 1e3
+            scan[f"2^{log2n}"] = {"us_per_call": us, "gbs": 32.0 * n_c / us / 1e3}
+            del P
+        out["retrieve_scan"] = scan
         return out
 
     def time_steps_e2e(self, steps: int):
@@ -498,6 +521,7 @@ def run_ours(args, w: wi.Workload):
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if w.name.startswith("cfg2") else None,
                      "kernel": "memory_attention_kernel"},
         "compress": side["compress"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
+        "retrieve_scan": side["retrieve_scan"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
     }

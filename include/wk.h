@@ -127,8 +127,8 @@ int64_t wk_pool_tag(const wk_ctx* ctx, int32_t slot); /* chunk_tag given at appe
 wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_t* slots_out_dev,
                       double* dist_out_dev, int32_t* n_out_host, void* stream);
 
-/* Query-based retrieval (Appendix C: stored chunks ranked "by their attention scores with respect to the current
- * denoising query"; the paper gives no formula).  Score of a stored chunk = the softmax mass the queries Q put on that
+/* Query-based retrieval (Appendix C ranks the stored chunks by how much attention the current denoising query pays
+ * them and gives no formula).  Score of a stored chunk = the softmax mass the queries Q put on that
  * chunk's stored keys of `layer` when they attend over all stored chunks, averaged over heads and query rows (scores
  * are >= 0 and sum to 1); the min(k, M) largest win, ties to the lowest slot, written in rank order.
  *   Q [lq][H][128] bf16; slots_out_dev [max_k] int32 (-1 past the count); score_out_dev [max_k] fp32 or NULL.
@@ -136,6 +136,22 @@ wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_
  * Errors: WK_ERR_SHAPE (lq > max_lq, k > max_k, layer out of range, pool_slots > 1024), WK_ERR_ARG, WK_ERR_UNBOUND. */
 wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, int32_t k, int32_t* slots_out_dev,
                             float* score_out_dev, int32_t* n_out_host, void* stream);
+
+/* World Retrieval over a plain pose array of any length (Eq. 4 with the distance of Section 5.1, same semantics as
+ * wk_retrieve: squared-L2 translation distance and geodesic rotation angle, each divided by its maximum over the valid
+ * candidates, summed, in fp64; the min(k, valid candidates) smallest win, ties to the lowest index, rank order).  For
+ * candidate sets far beyond a pool's slot table (the paper's pools hold 10^2..10^3 chunks; this call is what makes
+ * "GB/s of retrieval" measurable at 2^16..2^24 poses).  The poses are read twice: both maxima must be known before any
+ * distance can be formed.
+ *   poses_dev [n][8] fp32 (tx ty tz _ qw qx qy qz), 16-byte aligned; valid_dev [n] int32 or NULL (all valid);
+ *   cur_pose_host [8]; ids_out_dev [out_capacity] int32 (-1 past the count); dist_out_dev [out_capacity] fp64 or NULL;
+ *   scratch_dev: wk_retrieve_scan_scratch_bytes() bytes, 16-byte aligned, caller-owned, contents irrelevant on entry.
+ * ctx supplies the device, the SM count and the status word; its pool is not touched (an unbound context is fine).
+ * Errors: WK_ERR_SHAPE (k < 0, k > 64, k > out_capacity, n < 0 or n >= 2^31, scratch too small), WK_ERR_ARG. */
+size_t wk_retrieve_scan_scratch_bytes(void);
+wk_status wk_retrieve_scan(wk_ctx* ctx, const float* poses_dev, const int32_t* valid_dev, int64_t n,
+                           const float* cur_pose_host, int32_t k, int32_t* ids_out_dev, double* dist_out_dev,
+                           int32_t out_capacity, void* scratch_dev, size_t scratch_bytes, void* stream);
 
 /* The paper has no counterpart to this call: it exists for callers that may not allocate device memory.
  * Same computation and same results as wk_retrieve, but with no context and no caller-provided scratch: the two

@@ -66,6 +66,8 @@ def load_library() -> C.CDLL:
         "wk_pool_tag": (i64, [vp, i32]),
         "wk_retrieve": (i32, [vp, C.POINTER(C.c_float), i32, vp, vp, C.POINTER(i32), vp]),
         "wk_retrieve_query": (i32, [vp, i32, vp, i32, i32, vp, vp, C.POINTER(i32), vp]),
+        "wk_retrieve_scan_scratch_bytes": (C.c_size_t, []),
+        "wk_retrieve_scan": (i32, [vp, vp, vp, C.c_int64, C.POINTER(C.c_float), i32, vp, vp, i32, vp, C.c_size_t, vp]),
         "wk_retrieve_noalloc": (i32, [vp, vp, i32, C.POINTER(C.c_float), i32, i32, vp, vp, vp]),
         "wk_memory_attention": (i32, [vp, i32, vp, i32, C.POINTER(wk_dense_seg), i32, vp, i32, vp, vp, i32, vp]),
         "wk_poll_status": (i32, [vp, C.POINTER(C.c_uint32), vp]),
@@ -83,7 +85,7 @@ def load_library() -> C.CDLL:
 
 EXPORTED_SYMBOLS = ("wk_create", "wk_destroy", "wk_pool_bytes", "wk_scratch_bytes", "wk_bind", "wk_compress_chunk",
                     "wk_pool_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
-                    "wk_retrieve_noalloc", "wk_retrieve_query",
+                    "wk_retrieve_noalloc", "wk_retrieve_query", "wk_retrieve_scan", "wk_retrieve_scan_scratch_bytes",
                     "wk_memory_attention", "wk_poll_status", "wk_status_string", "wk_last_cuda_error",
                     "wk_launch_count")
 
@@ -212,6 +214,22 @@ class WorldKV:
         if st != WK_OK:
             raise WkError(st, "wk_retrieve")
         return slots_out, n_out.value
+
+    def retrieve_scan(self, poses: torch.Tensor, cur_pose: Sequence[float], k: int, valid: Optional[torch.Tensor] = None,
+                      ids_out: Optional[torch.Tensor] = None, dist_out: Optional[torch.Tensor] = None,
+                      scratch: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        """Retrieval over a plain pose array [n, 8] fp32 of any length; returns ids_out int32 (-1 past the count)."""
+        if ids_out is None:
+            ids_out = torch.empty(max(1, k), dtype=torch.int32, device=self.device)
+        if scratch is None:
+            scratch = torch.empty(self.lib.wk_retrieve_scan_scratch_bytes(), dtype=torch.uint8, device=self.device)
+        pose_arr = (C.c_float * 8)(*[float(x) for x in cur_pose])
+        st = self.lib.wk_retrieve_scan(self.ctx, poses.data_ptr(), _ptr(valid), poses.shape[0], pose_arr, k,
+                                       ids_out.data_ptr(), _ptr(dist_out), ids_out.numel(), scratch.data_ptr(),
+                                       scratch.numel(), _stream(stream))
+        if st != WK_OK:
+            raise WkError(st, "wk_retrieve_scan")
+        return ids_out
 
     def retrieve_query(self, layer: int, Q: torch.Tensor, k: int, slots_out: Optional[torch.Tensor] = None,
                        score_out: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, int]:

@@ -317,6 +317,19 @@ wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_
   return launch_retrieve(ctx, cur_pose_host, k, slots_out_dev, dist_out_dev, static_cast<cudaStream_t>(stream));
 }
 
+size_t wk_retrieve_scan_scratch_bytes(void) { return retrieve_scan_scratch_bytes(); }
+
+wk_status wk_retrieve_scan(wk_ctx* ctx, const float* poses_dev, const int32_t* valid_dev, int64_t n,
+                           const float* cur_pose_host, int32_t k, int32_t* ids_out_dev, double* dist_out_dev,
+                           int32_t out_capacity, void* scratch_dev, size_t scratch_bytes, void* stream) {
+  if (!ctx || !cur_pose_host || !ids_out_dev || !scratch_dev || (n > 0 && !poses_dev)) return WK_ERR_ARG;
+  if (!aligned16(poses_dev) || !aligned16(scratch_dev)) return WK_ERR_ARG;
+  if (k < 0 || k > 64 || k > out_capacity || n < 0 || n >= (int64_t(1) << 31)) return WK_ERR_SHAPE;
+  if (scratch_bytes < retrieve_scan_scratch_bytes()) return WK_ERR_SHAPE;
+  return launch_retrieve_scan(ctx, poses_dev, valid_dev, n, cur_pose_host, k, ids_out_dev, dist_out_dev, out_capacity,
+                              scratch_dev, static_cast<cudaStream_t>(stream));
+}
+
 wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t lq, int32_t k, int32_t* slots_out_dev,
                             float* score_out_dev, int32_t* n_out_host, void* stream) {
   if (!ctx || !Q || !slots_out_dev || !n_out_host || lq < 1) return WK_ERR_ARG;

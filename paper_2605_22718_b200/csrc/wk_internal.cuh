@@ -118,6 +118,9 @@ wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfl
                         int64_t stride, const int32_t* keep_idx, cudaStream_t s);
 wk_status launch_slot_mark(wk_ctx* ctx, int slot, int valid, const float* pose, cudaStream_t s);
 wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out, cudaStream_t s);
+size_t retrieve_scan_scratch_bytes();
+wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* valid, int64_t n, const float* cur_pose,
+                               int k, int32_t* ids_out, double* dist_out, int out_capacity, void* scratch, cudaStream_t s);
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
                            cudaStream_t s, bool lse_only = false);
