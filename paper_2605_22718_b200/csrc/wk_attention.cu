@@ -203,6 +203,8 @@ __device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
 // P = 2^(s * scale - m) for one row of a tile: rounds to bf16, stores into tensor memory over S (64 columns), returns
 // the fp32 row sum.  Every exponential goes to the MUFU: moving a share of them to a polynomial on the FMA pipe was
 // measured slower here (one softmax warp per SM sub-partition is latency-bound, not MUFU-throughput-bound).
+// kStore = false (LSE-only launches): only the row sum is wanted, nothing is written.
+template <bool kStore>
 __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t scale2, uint64_t neg_m2, uint32_t tS) {
   uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
 #pragma unroll
@@ -219,9 +221,9 @@ __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t 
       else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
       else if ((i & 3) == 2) acc2 = add_f32x2(acc2, pp);
       else acc3 = add_f32x2(acc3, pp);
-      pk[i] = pack_bf16x2(p0, p1);
+      if (kStore) pk[i] = pack_bf16x2(p0, p1);
     }
-    tmem_st_x16(tS + c * 16, pk);
+    if (kStore) tmem_st_x16(tS + c * 16, pk);
   }
   float a, b;
   unpack_f32x2(add_f32x2(add_f32x2(acc0, acc1), add_f32x2(acc2, acc3)), a, b);
@@ -267,6 +269,9 @@ struct PieceWalker {
   }
 };
 
+// kLse = true is the LSE-only instantiation (query-based retrieval): no V, no P, no O; a softmax thread hands its S
+// buffer back as soon as the row is in registers, so the next Q K^T runs under the exponentials.
+template <bool kLse>
 __global__ void __launch_bounds__(kThreads, 1)
 memory_attention_kernel(const __grid_constant__ AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -334,7 +339,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             tma_load_3d(dk, &p.tm_kpool, &bars.k_full[sk], x, ti.row0, ti.z);
             tma_load_3d(dk + kHalfTileBytes, &p.tm_kpool, &bars.k_full[sk], x + 64, ti.row0, ti.z);
           }
-          if (p.lse_only) { ++jk; continue; }   // no P V product: V is not fetched
+          if (kLse) { ++jk; continue; }   // no P V product: V is not fetched
           if (!(ok = wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status))) break;
           mbar_expect_tx(&bars.v_full[st], kTileBytes);
           uint8_t* dv = sV + st * kTileBytes;
@@ -435,12 +440,12 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           const uint32_t ph = (g / kStagesV) & 1, phn = ((g + 1) / kStagesK) & 1;
           const bool more = j + 1 < n_eff;
           WK_PROF(10, blockIdx.x == 0);
-          if (!p.lse_only && !(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
+          if (!kLse && !(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
           WK_PROF(11, blockIdx.x == 0);
           if (!(ok = wait_or_abort(&bars.p_full[0], g & 1, &s_abort, p.status))) break;
           WK_PROF(12, blockIdx.x == 0);
           tc_fence_after();
-          if (!p.lse_only) issue_pv(0, st, j > 0);
+          if (!kLse) issue_pv(0, st, j > 0);
           mma_commit(&bars.o_done[0]);
           if (more) {
             WK_PROF(13, blockIdx.x == 0);
@@ -455,10 +460,10 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             if (!(ok = wait_or_abort(&bars.p_full[1], (g1 + j) & 1, &s_abort, p.status))) break;
             WK_PROF(16, blockIdx.x == 0);
             tc_fence_after();
-            if (!p.lse_only) issue_pv(1, st, j > 0);
+            if (!kLse) issue_pv(1, st, j > 0);
             mma_commit(&bars.o_done[1]);
           }
-          if (!p.lse_only) mma_commit(&bars.v_empty[st]);
+          if (!kLse) mma_commit(&bars.v_empty[st]);
           if (more) {
             if (q1) { issue_s(1, stn); mma_commit(&bars.s_full[1]); }
             mma_commit(&bars.k_empty[stn]);
@@ -523,6 +528,11 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             tc_wait_ld();
           }
           WK_PROF(2, blockIdx.x == 0 && tid == 0);
+          if (kLse) {   // S is in registers and nothing goes back into the buffer: release it now
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.p_full[wg]);
+          }
           const bool full_tile = nv == kTileKV;
           if (!full_tile) {   // rows past the end of the segment were zero-filled by TMA: mask them out
             c0 = c1 = c2 = c3 = -INFINITY;
@@ -555,8 +565,8 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           l *= alpha;
           const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
           WK_PROF(3, blockIdx.x == 0 && tid == 0);
-          l += exp_store_tile(s, scale2, neg_m2, tS);   // masked columns hold -inf and come out as 0
-          if (__any_sync(0xffffffffu, rescale)) {
+          l += exp_store_tile<!kLse>(s, scale2, neg_m2, tS);   // masked columns hold -inf and come out as 0
+          if (!kLse && __any_sync(0xffffffffu, rescale)) {
             // the previous P V product must have landed before O is touched
             if (!(ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status))) break;
             tc_fence_after();
@@ -571,10 +581,12 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
             }
           }
           WK_PROF(4, blockIdx.x == 0 && tid == 0);
-          tc_wait_st();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars.p_full[wg]);   // one arrival per warp: the wait above covered all 32 lanes' stores
+          if (!kLse) {
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars.p_full[wg]);   // one arrival per warp: the wait above covered all 32 lanes' stores
+          }
           WK_PROF(5, blockIdx.x == 0 && tid == 0);
           ++j;
           ++g;
@@ -590,14 +602,14 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t r[32];
-            if (j > 0) {
+            if (!kLse && j > 0) {
               tmem_ld_x32(tO + c * 32, r);
               tc_wait_ld();
             } else {
 #pragma unroll
               for (int i = 0; i < 32; ++i) r[i] = 0u;
             }
-            if (qrow < p.lq && !p.lse_only) {
+            if (!kLse && qrow < p.lq) {
               if (pc.slot < 0) {
                 uint4* dst = reinterpret_cast<uint4*>(p.O + (static_cast<int64_t>(qrow) * p.H + pc.h) * kHeadDim + c * 32);
 #pragma unroll
@@ -701,7 +713,9 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
                            cudaStream_t s, bool lse_only) {
   static bool attr_set = false;
   if (!attr_set) {
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kSmemBytes)));
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(kSmemBytes)));
     attr_set = true;
   }
@@ -786,7 +800,8 @@ wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int l
   if (G > W) G = W;
   const int max_slots = attention_partial_slots(p.H, ctx->max_lq, ctx->max_splits);
   if (!lse_only && 2 * G > max_slots) return WK_ERR_SHAPE;
-  memory_attention_kernel<<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p);
+  if (lse_only) memory_attention_kernel<true><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p);
+  else memory_attention_kernel<false><<<static_cast<unsigned>(G), kThreads, kSmemBytes, s>>>(p);
   if ((st = after_launch(ctx)) != WK_OK) return st;
   if (!lse_only && G != p.n_units) {   // some unit was cut
     const int64_t warps = static_cast<int64_t>(p.n_units) * kPairRows;
