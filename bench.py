@@ -531,6 +531,46 @@ def run_ours(args, w: wi.Workload):
     print(json.dumps(line), flush=True)
 
 
+def run_retention_sweep(args, w):
+    """Throughput against retention (the paper's retention ablation, Section 5.3, as a cost curve): the same chunk step
+    with n_keep in {0, T/4, T/2, T, 3T/2, 2T} kept non-anchor tokens per stored chunk, i.e. stored chunks of
+    T + n_keep rows.  One JSON line with one point per rung; the pool holds 2k chunks (the step's traffic does not
+    depend on how many more are stored)."""
+    import dataclasses
+    import torch
+    rank, local, world = dist_env()
+    if rank != 0:
+        return
+    T = w.T
+    points = []
+    for nk in (0, T // 4, T // 2, T, 3 * T // 2, 2 * T):
+        w2 = dataclasses.replace(w, n_keep=nk, pool_chunks=2 * max(w.k, 1), name=f"{w.name}_keep{nk}")
+        b = ChunkStepBench(w2, local, e2e=False, kv_splits=args.kv_splits)
+        for _ in range(max(3, args.warmup)):
+            b.step()
+        b.attn_events = []
+        ms = b.time_steps(args.steps)
+        attn_ms = statistics.mean(e0.elapsed_time(e1) for e0, e1 in b.attn_events) / b.attention_calls_per_step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(10):
+            b.kv.compress_chunk(b.evK[i % len(b.evK)], keep_idx_out=b.keep)
+        e1.record()
+        torch.cuda.synchronize(b.dev)
+        st, flags = b.kv.poll_status()
+        if st != 0:
+            raise RuntimeError(f"device status {st} flags {flags}")
+        points.append({"n_keep": nk, "retention": (T + nk) / (w.F * T), "stored_rows_per_chunk": T + nk, "lkv": w2.Lkv,
+                       "chunk_step_ms": ms / args.steps, "attention_us_per_call": attn_ms * 1e3,
+                       "attention_tflops": w2.attention_flops() / (attn_ms * 1e-3) / 1e12,
+                       "compress_us_per_call": e0.elapsed_time(e1) / 10 * 1e3,
+                       "pool_bytes_per_chunk": 2 * w.n_layers * (T + nk) * w.D * 2})
+        del b
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "chunk-step cost against retention", "unit": "ms", "workload": w.name, "steps": args.steps,
+                      "k": w.k, "data": "synthetic", "points": points}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -543,11 +583,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profiler-range", action="store_true", help="bracket the timed steps with cudaProfilerStart/Stop")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--retention-sweep", action="store_true",
+                    help="instead of the bench line: chunk-step cost for n_keep in {0, T/4, T/2, T, 3T/2, 2T}")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = wi.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.retention_sweep:
+        run_retention_sweep(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)
