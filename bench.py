@@ -532,7 +532,7 @@ def run_ours(args, w: wi.Workload):
 
 
 def run_retention_sweep(args, w):
-    """Throughput against retention (the paper's retention ablation, Section 5.3, as a cost curve): the same chunk step
+    """Throughput against retention (the intra-chunk compression ratios of the ablation in Section 5.4, as a cost curve): the same chunk step
     with n_keep in {0, T/4, T/2, T, 3T/2, 2T} kept non-anchor tokens per stored chunk, i.e. stored chunks of
     T + n_keep rows.  One JSON line with one point per rung; the pool holds 2k chunks (the step's traffic does not
     depend on how many more are stored)."""
