@@ -116,6 +116,26 @@ int32_t wk_pool_oldest(const wk_ctx* ctx);   /* valid slot with the earliest app
 int32_t wk_pool_count(const wk_ctx* ctx);    /* number of valid slots */
 int64_t wk_pool_tag(const wk_ctx* ctx, int32_t slot); /* chunk_tag given at append, -1 if not valid */
 
+/* ---- host-memory tier (Section 7: every stored chunk in CPU memory, only the chunks the current attention needs on
+ *      the GPU; the paper leaves hiding the transfer to future work) ---------------------------------------------- */
+
+/* Bytes of one stored chunk in host memory: K then V, each [n_layers][T + n_keep][D] bf16. */
+size_t wk_host_chunk_bytes(const wk_ctx* ctx);
+
+/* Copies the chunk held by a visible slot to host memory in the layout above: two strided device-to-host copies on
+ * `stream`, asynchronous when host_dst is page-locked.  The slot stays as it is (evict it afterwards to free it).
+ * Errors: WK_ERR_BAD_SLOT (slot not visible), WK_ERR_ARG, WK_ERR_UNBOUND, WK_ERR_CUDA. */
+wk_status wk_pool_store_host(wk_ctx* ctx, int32_t slot, void* host_dst, void* stream);
+
+/* Brings layers layer0 .. layer0+n-1 of a chunk written by wk_pool_store_host back into the pool: into the lowest free
+ * slot on the first call (slot_io_host = -1 on entry, the slot is returned), into that slot on later calls, exactly as
+ * wk_pool_append does; the slot becomes visible, with the given pose, once every layer has been loaded.  Loading layer
+ * by layer lets the copy of layer l + 1 run under the attention of layer l.  host_src points at the start of the chunk's
+ * host image (not at the layer); copies run on `stream`.
+ * Errors: WK_ERR_POOL_FULL, WK_ERR_BAD_SLOT, WK_ERR_SHAPE, WK_ERR_ARG, WK_ERR_UNBOUND, WK_ERR_CUDA. */
+wk_status wk_pool_load_host(wk_ctx* ctx, int32_t layer0, int32_t n, const void* host_src, const float* pose_host,
+                            int64_t chunk_tag, int32_t* slot_io_host, void* stream);
+
 /* ---- World Retrieval (Section 4.2 Eq. 4; Section 5.1) -------------------------------------- */
 
 /* Distance of every stored chunk's pose to cur_pose: squared-L2 translation distance and geodesic

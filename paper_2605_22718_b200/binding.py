@@ -66,6 +66,9 @@ def load_library() -> C.CDLL:
         "wk_pool_tag": (i64, [vp, i32]),
         "wk_retrieve": (i32, [vp, C.POINTER(C.c_float), i32, vp, vp, C.POINTER(i32), vp]),
         "wk_retrieve_query": (i32, [vp, i32, vp, i32, i32, vp, vp, C.POINTER(i32), vp]),
+        "wk_host_chunk_bytes": (C.c_size_t, [vp]),
+        "wk_pool_store_host": (i32, [vp, i32, vp, vp]),
+        "wk_pool_load_host": (i32, [vp, i32, i32, vp, C.POINTER(C.c_float), C.c_int64, C.POINTER(i32), vp]),
         "wk_retrieve_scan_scratch_bytes": (C.c_size_t, []),
         "wk_retrieve_scan": (i32, [vp, vp, vp, C.c_int64, C.POINTER(C.c_float), i32, vp, vp, i32, vp, C.c_size_t, vp]),
         "wk_retrieve_noalloc": (i32, [vp, vp, i32, C.POINTER(C.c_float), i32, i32, vp, vp, vp]),
@@ -86,6 +89,7 @@ def load_library() -> C.CDLL:
 EXPORTED_SYMBOLS = ("wk_create", "wk_destroy", "wk_pool_bytes", "wk_scratch_bytes", "wk_bind", "wk_compress_chunk",
                     "wk_pool_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
                     "wk_retrieve_noalloc", "wk_retrieve_query", "wk_retrieve_scan", "wk_retrieve_scan_scratch_bytes",
+                    "wk_host_chunk_bytes", "wk_pool_store_host", "wk_pool_load_host",
                     "wk_memory_attention", "wk_poll_status", "wk_status_string", "wk_last_cuda_error",
                     "wk_launch_count")
 
@@ -214,6 +218,29 @@ class WorldKV:
         if st != WK_OK:
             raise WkError(st, "wk_retrieve")
         return slots_out, n_out.value
+
+    # ---- host-memory tier ----------------------------------------------------------------------
+    def host_chunk_bytes(self) -> int:
+        return self.lib.wk_host_chunk_bytes(self.ctx)
+
+    def pool_store_host(self, slot: int, host_dst: torch.Tensor, stream=None) -> None:
+        """Copies the chunk in `slot` into a (page-locked) host tensor of host_chunk_bytes() bytes."""
+        assert not host_dst.is_cuda and host_dst.numel() * host_dst.element_size() >= self.host_chunk_bytes()
+        st = self.lib.wk_pool_store_host(self.ctx, slot, host_dst.data_ptr(), _stream(stream))
+        if st != WK_OK:
+            raise WkError(st, "wk_pool_store_host")
+
+    def pool_load_host(self, layer0: int, n: int, host_src: torch.Tensor, pose: Sequence[float], chunk_tag: int = -1,
+                       slot: int = -1, stream=None) -> int:
+        """Loads layers [layer0, layer0 + n) of a host chunk image into the pool; returns the slot."""
+        assert not host_src.is_cuda and host_src.numel() * host_src.element_size() >= self.host_chunk_bytes()
+        pose_arr = (C.c_float * 8)(*[float(x) for x in pose])
+        slot_io = C.c_int32(slot)
+        st = self.lib.wk_pool_load_host(self.ctx, layer0, n, host_src.data_ptr(), pose_arr, chunk_tag, C.byref(slot_io),
+                                        _stream(stream))
+        if st != WK_OK:
+            raise WkError(st, "wk_pool_load_host")
+        return slot_io.value
 
     def retrieve_scan(self, poses: torch.Tensor, cur_pose: Sequence[float], k: int, valid: Optional[torch.Tensor] = None,
                       ids_out: Optional[torch.Tensor] = None, dist_out: Optional[torch.Tensor] = None,

@@ -275,6 +275,75 @@ wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_c
   return WK_OK;
 }
 
+size_t wk_host_chunk_bytes(const wk_ctx* ctx) {
+  if (!ctx) return 0;
+  return 2 * static_cast<size_t>(ctx->cfg.n_layers) * ctx->C * ctx->D * sizeof(__nv_bfloat16);
+}
+
+wk_status wk_pool_store_host(wk_ctx* ctx, int32_t slot, void* host_dst, void* stream) {
+  if (!ctx || !host_dst) return WK_ERR_ARG;
+  if (!ctx->bound) return WK_ERR_UNBOUND;
+  if (slot < 0 || slot >= ctx->cfg.pool_slots || ctx->slots[slot].state != SLOT_VALID) return WK_ERR_BAD_SLOT;
+  // one layer of one slot is contiguous (C * D elements); the layers of a slot are pool_slots such blocks apart
+  const size_t row = static_cast<size_t>(ctx->C) * ctx->D * sizeof(__nv_bfloat16);
+  const size_t pitch = row * ctx->cfg.pool_slots;
+  const int L = ctx->cfg.n_layers;
+  uint8_t* dst = static_cast<uint8_t*>(host_dst);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  WK_CUDA_TRY(ctx, cudaMemcpy2DAsync(dst, row, reinterpret_cast<const uint8_t*>(ctx->Kpool) + slot * row, pitch, row, L,
+                                     cudaMemcpyDeviceToHost, s));
+  WK_CUDA_TRY(ctx, cudaMemcpy2DAsync(dst + row * L, row, reinterpret_cast<const uint8_t*>(ctx->Vpool) + slot * row, pitch,
+                                     row, L, cudaMemcpyDeviceToHost, s));
+  return WK_OK;
+}
+
+wk_status wk_pool_load_host(wk_ctx* ctx, int32_t layer0, int32_t n, const void* host_src, const float* pose_host,
+                            int64_t chunk_tag, int32_t* slot_io_host, void* stream) {
+  if (!ctx || !host_src || !pose_host || !slot_io_host) return WK_ERR_ARG;
+  if (!ctx->bound) return WK_ERR_UNBOUND;
+  if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers) return WK_ERR_SHAPE;
+  int slot = *slot_io_host;
+  if (slot < 0) {
+    if (slot != -1) return WK_ERR_BAD_SLOT;
+    for (int s = 0; s < ctx->cfg.pool_slots; ++s) {
+      if (ctx->slots[s].state == SLOT_FREE) { slot = s; break; }
+    }
+    if (slot < 0) return WK_ERR_POOL_FULL;
+  } else {
+    if (slot >= ctx->cfg.pool_slots || ctx->slots[slot].state != SLOT_OPEN) return WK_ERR_BAD_SLOT;
+  }
+  SlotInfo& si = ctx->slots[slot];
+  for (int l = layer0; l < layer0 + n; ++l) {
+    if (si.state == SLOT_OPEN && si.layer_mask[l]) return WK_ERR_BAD_SLOT;  // layer loaded twice
+  }
+  const size_t row = static_cast<size_t>(ctx->C) * ctx->D * sizeof(__nv_bfloat16);
+  const size_t pitch = row * ctx->cfg.pool_slots;
+  const int L = ctx->cfg.n_layers;
+  const uint8_t* src = static_cast<const uint8_t*>(host_src);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  WK_CUDA_TRY(ctx, cudaMemcpy2DAsync(reinterpret_cast<uint8_t*>(ctx->Kpool) + layer0 * pitch + slot * row, pitch,
+                                     src + layer0 * row, row, row, n, cudaMemcpyHostToDevice, s));
+  WK_CUDA_TRY(ctx, cudaMemcpy2DAsync(reinterpret_cast<uint8_t*>(ctx->Vpool) + layer0 * pitch + slot * row, pitch,
+                                     src + (static_cast<size_t>(L) + layer0) * row, row, row, n, cudaMemcpyHostToDevice, s));
+  if (si.state == SLOT_FREE) {
+    si.state = SLOT_OPEN;
+    si.layers_done = 0;
+    si.layer_mask.assign(ctx->cfg.n_layers, 0);
+    si.tag = chunk_tag;
+    memcpy(si.pose, pose_host, sizeof(si.pose));
+  }
+  for (int l = layer0; l < layer0 + n; ++l) si.layer_mask[l] = 1;
+  si.layers_done += n;
+  if (si.layers_done == ctx->cfg.n_layers) {
+    wk_status st = launch_slot_mark(ctx, slot, 1, si.pose, s);
+    if (st != WK_OK) return st;
+    si.state = SLOT_VALID;
+    si.seq = ctx->next_seq++;
+  }
+  *slot_io_host = slot;
+  return WK_OK;
+}
+
 wk_status wk_pool_evict(wk_ctx* ctx, int32_t slot, void* stream) {
   if (!ctx) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
