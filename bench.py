@@ -125,7 +125,8 @@ def barrier():
 class ChunkStepBench:
     """Holds the pool, the per-layer window buffers and rotating inputs of one workload, and runs chunk steps."""
 
-    def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True, kv_splits: int = 0):
+    def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True, kv_splits: int = 0,
+                 prefill: bool = True):
         import torch
         from paper_2605_22718_b200 import WorldKV
         from wkinputs import device as wd
@@ -149,7 +150,7 @@ class ChunkStepBench:
         Kc = torch.empty((L, w.F * T, D), dtype=bf, device=self.dev)
         Vc = torch.empty((L, w.F * T, D), dtype=bf, device=self.dev)
         self.keep = torch.empty((L, w.C), dtype=torch.int32, device=self.dev)
-        for c in range(w.pool_chunks):
+        for c in range(w.pool_chunks if prefill else 0):
             for l in range(L):
                 wd.key_chunk(Kc[l], w.seed, l, c, T, D, w.sigma, w.F)
                 wd.value_chunk(Vc[l], w.seed, l, c, T, D, w.F)
@@ -531,6 +532,130 @@ def run_ours(args, w: wi.Workload):
     print(json.dumps(line), flush=True)
 
 
+def run_host_tier(args, w):
+    """The chunk step with every stored chunk in page-locked host memory (the paper's CPU-offloading direction, Section 7):
+    the device pool holds only two sets of k slots.  While step i computes, the k chunks step i + 1 will attend to are
+    picked by pose over the host tier's pose table (wk_retrieve_scan) and loaded on a copy stream; the chunk leaving the
+    window is compressed, appended, copied out to the host tier and evicted.  The poses of the rollout are scripted, so
+    the next pose is known one step ahead; in a live rollout it is the pending action's pose.  One JSON line."""
+    import dataclasses
+    import torch
+    rank, local, world = dist_env()
+    if rank != 0:
+        return
+    k = max(w.k, 1)
+    n_host = 4 * k
+    w2 = dataclasses.replace(w, pool_chunks=2 * k + 2, name=f"{w.name}_host_tier")
+    b = ChunkStepBench(w2, local, e2e=False, kv_splits=args.kv_splits, prefill=False)
+    kv, dev = b.kv, b.dev
+    L, T, D = w.n_layers, w.T, w.D
+    nbytes = kv.host_chunk_bytes()
+    host = [torch.empty(nbytes // 2, dtype=torch.int16).pin_memory() for _ in range(n_host + 1)]
+    host_pose = torch.zeros((n_host, 8), dtype=torch.float32)
+    comp, copy, out = torch.cuda.current_stream(dev), torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    # fill the host tier through the product path: generate -> compress -> append -> copy out -> evict
+    Kc, Vc = b.evK[0], b.evV[0]
+    for c in range(n_host):
+        for l in range(L):
+            b.wd.key_chunk(Kc[l], w.seed, l, c, T, D, w.sigma, w.F)
+            b.wd.value_chunk(Vc[l], w.seed, l, c, T, D, w.F)
+        kv.compress_chunk(Kc, keep_idx_out=b.keep)
+        slot = kv.pool_append(0, L, Kc, Vc, b.keep, b.poses[c], chunk_tag=c)
+        kv.pool_store_host(slot, host[c])
+        kv.pool_evict(slot)
+        host_pose[c] = torch.from_numpy(np.asarray(b.poses[c], dtype=np.float32))
+    torch.cuda.synchronize(dev)
+    pose_dev = host_pose.to(dev)
+    # transfer rates of one chunk image, each direction on its own
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(4):
+        s = kv.pool_load_host(0, L, host[i], b.poses[i])
+        kv.pool_evict(s)
+    e1.record()
+    torch.cuda.synchronize(dev)
+    h2d_gbs = 4 * nbytes / e0.elapsed_time(e1) / 1e6
+    s = kv.pool_load_host(0, L, host[0], b.poses[0])
+    e0.record()
+    for i in range(4):
+        kv.pool_store_host(s, host[n_host])
+    e1.record()
+    torch.cuda.synchronize(dev)
+    kv.pool_evict(s)
+    d2h_gbs = 4 * nbytes / e0.elapsed_time(e1) / 1e6
+    ids_dev = torch.empty(k, dtype=torch.int32, device=dev)
+    scratch = torch.empty(kv.lib.wk_retrieve_scan_scratch_bytes(), dtype=torch.uint8, device=dev)
+    sets = [[], []]                      # device slots of the two chunk sets
+    slot_lists = [torch.full((k,), -1, dtype=torch.int32, device=dev) for _ in range(2)]
+    loaded = [None, None]                # event: set i is on the device
+    done = [None, None]                  # event: the step that used set i has finished
+    stored = [None, -1]                  # event: the last copy-out has left its slot; that slot (kept until then)
+
+    def fetch(step: int):
+        """Pick and load the chunks of `step` into set step % 2 (copy stream)."""
+        j = step % 2
+        with torch.cuda.stream(copy):
+            if done[j] is not None:
+                copy.wait_event(done[j])
+            for sl in sets[j]:
+                kv.pool_evict(sl, stream=copy)
+            pose = b.poses[(n_host + step) % len(b.poses)]
+            kv.retrieve_scan(pose_dev, pose, k, ids_out=ids_dev, scratch=scratch, stream=copy)
+            ids = ids_dev.cpu().tolist()                     # waits for the copy stream only
+            sets[j] = [kv.pool_load_host(0, L, host[c], host_pose[c].tolist(), chunk_tag=c, stream=copy) for c in ids if c >= 0]
+            slot_lists[j][:len(sets[j])] = torch.tensor(sets[j], dtype=torch.int32)
+            loaded[j] = torch.cuda.Event()
+            loaded[j].record(copy)
+
+    def step(i: int):
+        j = i % 2
+        comp.wait_event(loaded[j])
+        for st in range(w.denoise_steps):
+            for l in range(L):
+                segs = [(b.curK[l], b.curV[l])]
+                if w.window_frames > 0:
+                    segs.append((b.winK[l], b.winV[l]))
+                kv.memory_attention(l, b.Q[l, st], segs, slot_lists[j], len(sets[j]), O=b.O[l, st], kv_splits=args.kv_splits)
+        done[j] = torch.cuda.Event()
+        done[j].record(comp)
+        # the chunk leaving the window goes to the host tier, replacing its oldest chunk
+        e = i % len(b.evK)
+        if stored[0] is not None:        # the previous copy-out has finished: only now is its slot given back
+            comp.wait_event(stored[0])
+            kv.pool_evict(stored[1])
+        kv.compress_chunk(b.evK[e], keep_idx_out=b.keep)
+        slot = kv.pool_append(0, L, b.evK[e], b.evV[e], b.keep, b.poses[(n_host + i) % len(b.poses)], chunk_tag=n_host + i)
+        ev = torch.cuda.Event()
+        ev.record(comp)
+        with torch.cuda.stream(out):
+            out.wait_event(ev)
+            kv.pool_store_host(slot, host[n_host], stream=out)
+            stored[0] = torch.cuda.Event()
+            stored[0].record(out)
+            stored[1] = slot
+
+    fetch(0)
+    total = max(3, args.warmup) + args.steps
+    for i in range(total):
+        if i == max(3, args.warmup):
+            t0 = torch.cuda.Event(enable_timing=True)
+            t0.record(comp)
+        step(i)
+        fetch(i + 1)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t1.record(comp)
+    torch.cuda.synchronize(dev)
+    st, flags = kv.poll_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} flags {flags}")
+    ms = t0.elapsed_time(t1) / args.steps
+    flops = w.attention_flops() * b.attention_calls_per_step()
+    print(json.dumps({"metric": "chunk step with the stored chunks in host memory", "unit": "ms", "workload": w.name,
+                      "steps": args.steps, "chunk_step_ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+                      "host_chunks": n_host, "chunk_bytes": nbytes, "fetch_bytes_per_step": k * nbytes,
+                      "store_bytes_per_step": nbytes, "h2d_gbs": h2d_gbs, "d2h_gbs": d2h_gbs, "data": "synthetic"}))
+
+
 def run_retention_sweep(args, w):
     """Throughput against retention (the intra-chunk compression ratios of the ablation in Section 5.4, as a cost curve): the same chunk step
     with n_keep in {0, T/4, T/2, T, 3T/2, 2T} kept non-anchor tokens per stored chunk, i.e. stored chunks of
@@ -583,13 +708,17 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profiler-range", action="store_true", help="bracket the timed steps with cudaProfilerStart/Stop")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--host-tier", action="store_true",
+                    help="instead of the bench line: the chunk step with the stored chunks fetched from host memory")
     ap.add_argument("--retention-sweep", action="store_true",
                     help="instead of the bench line: chunk-step cost for n_keep in {0, T/4, T/2, T, 3T/2, 2T}")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     w = wi.WORKLOADS[args.workload]
-    if args.retention_sweep:
+    if args.host_tier:
+        run_host_tier(args, w)
+    elif args.retention_sweep:
         run_retention_sweep(args, w)
     elif args.impl == "reference":
         run_reference(args, w)
