@@ -125,6 +125,22 @@ def compress_chunk(K_chunk, T: int, n_keep: int, form: str = "factorised"):
     return idx, s, margin
 
 
+def compress_chunk_per_head(K_chunk, T: int, n_keep: int, n_heads: int, form: str = "factorised"):
+    """The other reading of Eq. 5's key vector: one attention head's key (d = head_dim) instead of the whole
+    per-layer key, hence one keep-set per (layer, chunk, head).  K_chunk: [F*T, n_heads*head_dim]; head h owns
+    columns [h*head_dim, (h+1)*head_dim).  Returns (keep_idx int32[n_heads][T+n_keep], scores [n_heads][(F-1)*T],
+    smallest margin over the heads)."""
+    Kf = np.asarray(K_chunk)
+    d = Kf.shape[1] // n_heads
+    idx, sc, margin = [], [], float("inf")
+    for h in range(n_heads):
+        i, s, m = compress_chunk(Kf[:, h * d:(h + 1) * d], T, n_keep, form)
+        idx.append(i)
+        sc.append(s)
+        margin = min(margin, m)
+    return np.stack(idx), np.stack(sc), margin
+
+
 # --------------------------------------------------------------------------------------
 # World Retrieval (Section 4.2 Eq. 4, Section 5.1 distance)
 # --------------------------------------------------------------------------------------
@@ -236,8 +252,13 @@ class PoolModel:
         s = free[0]
         for l in range(self.n_layers):
             idx = np.asarray(keep_idx_layers[l])
-            self.K[(l, s)] = np.asarray(K_layers[l])[idx]
-            self.V[(l, s)] = np.asarray(V_layers[l])[idx]
+            Kl, Vl = np.asarray(K_layers[l]), np.asarray(V_layers[l])
+            if idx.ndim == 1:
+                self.K[(l, s)] = Kl[idx]
+                self.V[(l, s)] = Vl[idx]
+            else:   # one keep-set per head: stored row c of head h is token idx[h][c] of that head
+                self.K[(l, s)] = np.stack([Kl[idx[h], h] for h in range(idx.shape[0])], axis=1)
+                self.V[(l, s)] = np.stack([Vl[idx[h], h] for h in range(idx.shape[0])], axis=1)
         self.pose[s] = np.asarray(pose, dtype=np.float32).copy()
         self.seq[s] = self._next_seq
         self.tag[s] = tag

@@ -198,3 +198,71 @@ def test_redrawn_positions_are_enriched_in_the_keep_set():
     redrawn = np.concatenate([r1, r2])
     kept = idx[T:] - T
     assert redrawn[kept].mean() > redrawn.mean() + 0.05
+
+
+# ----------------------------------------------------------------------------- per-head keep-sets
+def _head_chunk(T=12, H=3, d=8, seed=0):
+    rng = np.random.default_rng(seed)
+    return rng.standard_normal((3 * T, H * d)), T, H, d
+
+
+def test_per_head_with_one_head_is_the_whole_key_reading():
+    K, T, H, d = _head_chunk(H=1)
+    idx, sc, m = o.compress_chunk_per_head(K, T, T // 2, 1)
+    idx0, sc0, m0 = o.compress_chunk(K, T, T // 2)
+    np.testing.assert_array_equal(idx[0], idx0)
+    np.testing.assert_array_equal(sc[0], sc0)
+    assert m == m0
+
+
+def test_per_head_scores_are_blind_to_the_other_heads():
+    """Brute force per head from the definition (mean cosine to every anchor key of that head), and: changing head 1's
+    columns leaves head 0's and head 2's keep-sets alone; permuting the heads permutes the keep-sets."""
+    K, T, H, d = _head_chunk()
+    idx, sc, _ = o.compress_chunk_per_head(K, T, 7, H)
+    for h in range(H):
+        Kh = K[:, h * d:(h + 1) * d]
+        A, N = Kh[:T], Kh[T:]
+        cos = (N / np.linalg.norm(N, axis=1, keepdims=True)) @ (A / np.linalg.norm(A, axis=1, keepdims=True)).T
+        np.testing.assert_allclose(sc[h], cos.mean(axis=1), atol=1e-14)
+        keep = np.sort(np.argsort(cos.mean(axis=1), kind="stable")[:7]) + T
+        np.testing.assert_array_equal(idx[h], np.concatenate([np.arange(T), keep]))
+    K2 = K.copy()
+    K2[:, d:2 * d] = np.random.default_rng(9).standard_normal((3 * T, d))
+    idx2, _, _ = o.compress_chunk_per_head(K2, T, 7, H)
+    np.testing.assert_array_equal(idx2[0], idx[0])
+    np.testing.assert_array_equal(idx2[2], idx[2])
+    assert not np.array_equal(idx2[1], idx[1])
+    perm = [2, 0, 1]
+    Kp = np.concatenate([K[:, p * d:(p + 1) * d] for p in perm], axis=1)
+    idxp, _, _ = o.compress_chunk_per_head(Kp, T, 7, H)
+    np.testing.assert_array_equal(idxp, idx[perm])
+
+
+def test_per_head_redundancy_is_found_head_by_head():
+    """Head 0 of the second frame repeats the anchor frame's head 0 (most similar to the anchors -> dropped first),
+    head 1 of the third frame does; each head drops its own redundant frame."""
+    rng = np.random.default_rng(4)
+    T, d = 10, 16
+    base = rng.standard_normal((T, d))
+    K = rng.standard_normal((3 * T, 2 * d))
+    K[:T, :d] = base + 5.0                      # a common offset makes anchor keys of head 0 alike
+    K[T:2 * T, :d] = base + 5.0                 # frame 1, head 0: copies of the anchors
+    K[:T, d:] = base - 5.0
+    K[2 * T:, d:] = base - 5.0                  # frame 2, head 1: copies of the anchors
+    idx, _, _ = o.compress_chunk_per_head(K, T, T, 2)
+    np.testing.assert_array_equal(idx[0][T:], np.arange(2 * T, 3 * T))   # head 0 keeps frame 2
+    np.testing.assert_array_equal(idx[1][T:], np.arange(T, 2 * T))       # head 1 keeps frame 1
+
+
+def test_pool_model_stores_per_head_rows():
+    K, T, H, d = _head_chunk()
+    V = np.random.default_rng(2).standard_normal(K.shape)
+    idx, _, _ = o.compress_chunk_per_head(K, T, 5, H)
+    pool = o.PoolModel(n_slots=2, n_layers=1)
+    s = pool.append([K.reshape(-1, H, d)], [V.reshape(-1, H, d)], [idx], wi.random_poses(0, 1)[0])
+    Ks = pool.K[(0, s)]
+    assert Ks.shape == (T + 5, H, d)
+    for h in range(H):
+        np.testing.assert_array_equal(Ks[:, h], K.reshape(-1, H, d)[idx[h], h])
+        np.testing.assert_array_equal(pool.V[(0, s)][:, h], V.reshape(-1, H, d)[idx[h], h])
