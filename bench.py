@@ -277,6 +277,23 @@ class ChunkStepBench:
         us = e0.elapsed_time(e1) / iters * 1e3
         nbytes = w.n_layers * w.F * w.T * w.D * 2
         out["compress"] = {"us_per_call": us, "bytes_per_call": nbytes, "gbs": nbytes / us / 1e3, "problems": w.n_layers}
+        # the same call with one keep-set per head (n_heads problems of 128 columns per chunk instead of one of D columns)
+        from paper_2605_22718_b200 import WorldKV, SCORE_PER_HEAD
+        kvh = WorldKV(n_layers=w.n_layers, n_heads=w.n_heads, tokens_per_frame=w.T, n_keep=w.n_keep, pool_slots=1, max_k=1,
+                      device=self.dev.index, max_batch=w.n_layers, score_mode=SCORE_PER_HEAD)
+        keep_h = torch.empty((w.n_layers, w.n_heads, w.C), dtype=torch.int32, device=self.dev)
+        for i in range(4):
+            kvh.compress_chunk(self.evK[i % len(self.evK)], keep_idx_out=keep_h)
+        torch.cuda.synchronize(self.dev)
+        e0.record()
+        for i in range(iters):
+            kvh.compress_chunk(self.evK[i % len(self.evK)], keep_idx_out=keep_h)
+        e1.record()
+        torch.cuda.synchronize(self.dev)
+        us = e0.elapsed_time(e1) / iters * 1e3
+        out["compress_per_head"] = {"us_per_call": us, "bytes_per_call": nbytes, "gbs": nbytes / us / 1e3,
+                                    "problems": w.n_layers * w.n_heads}
+        del kvh
         pose = self.poses[w.pool_chunks % len(self.poses)]
         e0.record()
         for i in range(iters):
@@ -521,7 +538,7 @@ def run_ours(args, w: wi.Workload):
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if w.name.startswith("cfg2") else None,
                      "kernel": "memory_attention_kernel"},
-        "compress": side["compress"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
+        "compress": side["compress"], "compress_per_head": side["compress_per_head"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
         "retrieve_scan": side["retrieve_scan"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,

@@ -62,8 +62,15 @@ typedef struct {
   int32_t max_dense_segments;/* 1..8 */
   int32_t device;            /* CUDA device ordinal */
   float softmax_scale;       /* 0 selects 1/sqrt(head_dim) */
-  int32_t reserved;          /* must be 0 */
+  int32_t score_mode;        /* WK_SCORE_WHOLE_KEY or WK_SCORE_PER_HEAD: what Eq. 5 takes as a token's key */
 } wk_config;
+
+/* Eq. 5 scores "keys"; the paper does not say whether that is the whole per-layer key of a token or one attention
+ * head's key.  Both readings are built:
+ *   WK_SCORE_WHOLE_KEY  all heads concatenated (d = n_heads * 128): one keep-set per (layer, chunk), shared by the heads
+ *   WK_SCORE_PER_HEAD   one head's key (d = 128): one keep-set per (layer, chunk, head); stored row c of head h is then
+ *                       token keep_idx[h][c] of that head, so the pool layout and the attention call do not change */
+enum { WK_SCORE_WHOLE_KEY = 0, WK_SCORE_PER_HEAD = 2 };
 
 /* ---- context ------------------------------------------------------------------------------- */
 
@@ -90,9 +97,11 @@ wk_status wk_bind(wk_ctx* ctx, void* pool_dev, size_t pool_bytes, void* scratch_
  * mean cosine similarity to the T anchor-frame keys (whole-token keys, all heads concatenated); the
  * n_keep lowest pooled scores are kept, ties to the lowest index.
  *   K_chunks     [batch] problems, problem b at K_chunks + b * batch_stride_elems, each [F*T][D] bf16
- *   keep_idx_out [batch][T + n_keep] int32: chunk-local token indices, ascending (anchors 0..T-1 first)
- *   scores_out   [batch][(F-1)*T] fp32 or NULL: the fp32 first-pass scores, for inspection only;
- *                the selection itself is decided on fp64 values near the threshold
+ *   keep_idx_out [batch][T + n_keep] int32: chunk-local token indices, ascending (anchors 0..T-1 first);
+ *                with WK_SCORE_PER_HEAD [batch][n_heads][T + n_keep], the score of a token then being taken on the
+ *                128 columns of that head alone
+ *   scores_out   [batch][(F-1)*T] fp32 ([batch][n_heads][(F-1)*T] per head) or NULL: the fp32 first-pass scores, for
+ *                inspection only; the selection itself is decided on fp64 values near the threshold
  * Errors: WK_ERR_ARG, WK_ERR_SHAPE (batch > max_batch), WK_ERR_UNBOUND. */
 wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_stride_elems, int32_t batch,
                             int32_t* keep_idx_out, float* scores_out, void* stream);
@@ -105,7 +114,8 @@ wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_str
  * ranges: the first call (slot_io_host = -1 on entry) picks the slot and returns it; later calls pass it
  * back.  The slot becomes visible to wk_retrieve / wk_memory_attention once every layer is stored.
  *   K_chunks, V_chunks  layer l at + (l - layer0) * batch_stride_elems, each [F*T][D] bf16
- *   keep_idx_dev        [n][T + n_keep] int32 (the output of wk_compress_chunk)
+ *   keep_idx_dev        [n][T + n_keep] int32, or [n][n_heads][T + n_keep] with WK_SCORE_PER_HEAD (the output of
+ *                       wk_compress_chunk)
  * Errors: WK_ERR_POOL_FULL, WK_ERR_BAD_SLOT (slot_io_host not an open append), WK_ERR_SHAPE, WK_ERR_ARG. */
 wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
                          int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,

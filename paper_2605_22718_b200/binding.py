@@ -25,11 +25,14 @@ class wk_config(C.Structure):
     _fields_ = [("n_layers", C.c_int32), ("n_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("tokens_per_frame", C.c_int32), ("frames_per_chunk", C.c_int32), ("n_keep", C.c_int32),
                 ("pool_slots", C.c_int32), ("max_k", C.c_int32), ("max_dense_segments", C.c_int32),
-                ("device", C.c_int32), ("softmax_scale", C.c_float), ("reserved", C.c_int32)]
+                ("device", C.c_int32), ("softmax_scale", C.c_float), ("score_mode", C.c_int32)]
 
 
 class wk_dense_seg(C.Structure):
     _fields_ = [("K", C.c_void_p), ("V", C.c_void_p), ("n_tokens", C.c_int32), ("reserved", C.c_int32)]
+
+
+SCORE_WHOLE_KEY, SCORE_PER_HEAD = 0, 2     # wk_config.score_mode
 
 
 class WkError(RuntimeError):
@@ -127,10 +130,11 @@ class WorldKV:
 
     def __init__(self, n_layers: int, n_heads: int, tokens_per_frame: int, n_keep: int, pool_slots: int, max_k: int,
                  frames_per_chunk: int = 3, max_dense_segments: int = 4, device: int = 0, softmax_scale: float = 0.0,
-                 max_batch: int = 1, max_lq: int = 0, max_splits: int = 1):
+                 max_batch: int = 1, max_lq: int = 0, max_splits: int = 1, score_mode: int = 0):
         self.lib = load_library()
         self.cfg = wk_config(n_layers, n_heads, 128, tokens_per_frame, frames_per_chunk, n_keep, pool_slots, max_k,
-                             max_dense_segments, device, softmax_scale, 0)
+                             max_dense_segments, device, softmax_scale, score_mode)
+        self.score_mode, self.n_heads = score_mode, n_heads
         self.T, self.F, self.H, self.D = tokens_per_frame, frames_per_chunk, n_heads, n_heads * 128
         self.C = tokens_per_frame + n_keep
         self.NA = (frames_per_chunk - 1) * tokens_per_frame
@@ -164,13 +168,15 @@ class WorldKV:
     def compress_chunk(self, K_chunks: torch.Tensor, keep_idx_out: Optional[torch.Tensor] = None,
                        scores_out: Optional[torch.Tensor] = None, batch: Optional[int] = None,
                        batch_stride_elems: Optional[int] = None, stream=None) -> torch.Tensor:
-        """K_chunks: [batch, F*T, D] bf16.  Returns keep_idx [batch, T + n_keep] int32."""
+        """K_chunks: [batch, F*T, D] bf16.  Returns keep_idx [batch, T + n_keep] int32 ([batch, H, T + n_keep] with
+        per-head keep-sets)."""
         if batch is None:
             batch = K_chunks.shape[0] if K_chunks.dim() == 3 else 1
         if batch_stride_elems is None:
             batch_stride_elems = K_chunks.stride(0) if K_chunks.dim() == 3 else self.F * self.T * self.D
         if keep_idx_out is None:
-            keep_idx_out = torch.empty((batch, self.C), dtype=torch.int32, device=self.device)
+            shape = (batch, self.n_heads, self.C) if self.score_mode == SCORE_PER_HEAD else (batch, self.C)
+            keep_idx_out = torch.empty(shape, dtype=torch.int32, device=self.device)
         st = self.lib.wk_compress_chunk(self.ctx, K_chunks.data_ptr(), batch_stride_elems, batch,
                                         keep_idx_out.data_ptr(), _ptr(scores_out), _stream(stream))
         if st != WK_OK:

@@ -26,14 +26,17 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   ScratchLayout s;
   const size_t D = static_cast<size_t>(c.n_heads) * c.head_dim;
   const size_t NA = static_cast<size_t>(c.frames_per_chunk - 1) * c.tokens_per_frame;
-  const size_t B = static_cast<size_t>(max_batch > 0 ? max_batch : 1);
+  // per-head scoring makes n_heads problems of 128 columns out of every chunk: the column-sized arrays keep their
+  // size, the per-problem ones grow by n_heads
+  const size_t Bc = static_cast<size_t>(max_batch > 0 ? max_batch : 1);
+  const size_t B = Bc * (c.score_mode == WK_SCORE_PER_HEAD ? c.n_heads : 1);
   s.anchor_parts = 16;
   size_t off = 0;
-  s.m32_off = off;   off += align_up(B * D * sizeof(float), 256);
-  s.m64_off = off;   off += align_up(B * D * sizeof(double), 256);
+  s.m32_off = off;   off += align_up(Bc * D * sizeof(float), 256);
+  s.m64_off = off;   off += align_up(Bc * D * sizeof(double), 256);
   s.s32_off = off;   off += align_up(B * NA * sizeof(float), 256);
   s.mnorm_off = off; off += align_up(B * 32 * sizeof(double), 256);   // up to 32 shares of |m|^2 per problem
-  s.part_off = off;  off += align_up(B * s.anchor_parts * D * sizeof(double), 256);
+  s.part_off = off;  off += align_up(Bc * s.anchor_parts * D * sizeof(double), 256);
   s.inv_off = off;   off += align_up(B * c.tokens_per_frame * sizeof(double), 256);
   s.cnt_off = off;   off += align_up(B * sizeof(uint32_t), 256);
   s.dist_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * 2 * sizeof(double), 256);
@@ -131,7 +134,8 @@ static wk_status check_config(const wk_config* c) {
   if (c->n_keep < 0 || c->n_keep > (c->frames_per_chunk - 1) * c->tokens_per_frame) return WK_ERR_ARG;
   if (c->pool_slots < 1 || c->max_k < 0) return WK_ERR_ARG;
   if (c->max_dense_segments < 1 || c->max_dense_segments > kMaxDenseSegs) return WK_ERR_ARG;
-  if (c->reserved != 0 || !(c->softmax_scale >= 0.f)) return WK_ERR_ARG;
+  if ((c->score_mode != WK_SCORE_WHOLE_KEY && c->score_mode != WK_SCORE_PER_HEAD) || !(c->softmax_scale >= 0.f))
+    return WK_ERR_ARG;
   if (static_cast<int64_t>(c->n_layers) * c->pool_slots > 0x7fffffffLL) return WK_ERR_ARG;
   return WK_OK;
 }

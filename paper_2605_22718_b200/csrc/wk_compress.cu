@@ -45,6 +45,18 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// Where the rows of problem b live.  A chunk is [F*T][rs] bf16; with whole-token keys (one keep-set per chunk) a
+// problem is a chunk and D = rs; with per-head keys a chunk holds hs = n_heads problems, problem (chunk, h) owning
+// columns [h*D, (h+1)*D) of every row, D = head_dim.
+struct RowMap {
+  int64_t stride;   // elements between chunks
+  int rs;           // elements between token rows
+  int hs;           // problems per chunk
+  __device__ __forceinline__ const __nv_bfloat16* base(const __nv_bfloat16* K, int b, int D) const {
+    return K + static_cast<int64_t>(b / hs) * stride + static_cast<int64_t>(b % hs) * D;
+  }
+};
+
 // ------------------------------------------------------------------------------------------------
 // anchor pass, two streaming kernels with no block barrier in their loops.
 //   anchor_norms:      one warp per anchor row, fp64 squared norm -> 1/|a_i| (0 for a zero key)
@@ -53,12 +65,12 @@ __device__ __forceinline__ float warp_sum(float v) {
 //                      time.  The last CTA of a problem adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kAnchorThreads)
-anchor_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, double* __restrict__ inv_norm) {
+anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, double* __restrict__ inv_norm) {
   const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
   if (r >= T) return;
   const int vecs = D >> 3;
-  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(r) * D);
+  const uint4* row = reinterpret_cast<const uint4*>(rm.base(K, b, D) + static_cast<int64_t>(r) * rm.rs);
   double n2a = 0.0, n2b = 0.0;
   for (int v0 = lane; v0 < vecs; v0 += 128) {
     uint4 q[4];
@@ -80,13 +92,14 @@ anchor_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, 
 }
 
 __global__ void __launch_bounds__(512)
-anchor_accumulate(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int parts,
+anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, int parts,
                   const double* __restrict__ inv_norm, double* __restrict__ partial) {
   const int b = blockIdx.y, part = blockIdx.x / kColSplit, csplit = blockIdx.x % kColSplit;
   const int tid = threadIdx.x, nthreads = blockDim.x;
   const int vecs = D >> 3;
   const int vec = csplit * nthreads + tid;   // the 16-byte column group this thread owns
-  const uint4* Kb = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride);
+  const uint4* Kb = reinterpret_cast<const uint4*>(rm.base(K, b, D));
+  const int64_t rsv = rm.rs >> 3;   // row pitch in 16-byte vectors
   const double* inv = inv_norm + static_cast<int64_t>(b) * T;
   if (vec < vecs) {
     double acc[8];
@@ -99,7 +112,7 @@ anchor_accumulate(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, in
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const int r = r0 + u * parts;
-        q[u] = r < T ? __ldg(Kb + static_cast<int64_t>(r) * vecs + vec) : make_uint4(0, 0, 0, 0);
+        q[u] = r < T ? __ldg(Kb + static_cast<int64_t>(r) * rsv + vec) : make_uint4(0, 0, 0, 0);
         sc[u] = r < T ? __ldg(inv + r) : 0.0;
       }
 #pragma unroll
@@ -225,7 +238,7 @@ anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int
 // shuffle additions; select_pass derives its error band from exactly this order.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kScoreThreads)
-score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D,
+score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
            const float* __restrict__ m32, float* __restrict__ s32, float* __restrict__ scores_out,
            uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
@@ -237,14 +250,14 @@ score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
   const int vecs = D >> 3;
   const int j0 = blockIdx.x * kScoreRowsPerCta;
   const int j1 = min(NA, j0 + kScoreRowsPerCta);
-  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * D;
+  const __nv_bfloat16* Kb = rm.base(K, b, D) + static_cast<int64_t>(T) * rm.rs;
   // two rows per warp at a time, so that twice as many 16-byte loads are in flight
   constexpr int W = kScoreThreads / 32;
   for (int j = j0 + warp; j < j1; j += 2 * W) {
     const int jb = j + W;
     const bool has_b = jb < j1;
-    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
-    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * D);
+    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * rm.rs);
+    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * rm.rs);
     float dot_a = 0.f, n2_a = 0.f, dot_b = 0.f, n2_b = 0.f;
     for (int v0 = lane; v0 < vecs; v0 += 128) {
       uint4 qa[4], qb[4];
@@ -299,7 +312,7 @@ __device__ __forceinline__ float key_f32(uint32_t k) {
 }
 
 __global__ void __launch_bounds__(kSelectThreads)
-select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int n_keep,
+select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D, int n_keep,
             const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
             int n_norm_parts, int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
@@ -385,7 +398,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
   const int need = n_keep - static_cast<int>(n_below);   // >= 1: the threshold token itself is in the band
   // exact fp64 scores of the band tokens: the whole CTA works on four tokens at a time (thread = one 16-byte vector
   // of the row), partial sums meet in shared memory and are added in a fixed order
-  const __nv_bfloat16* Nb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * D;
+  const __nv_bfloat16* Nb = rm.base(K, b, D) + static_cast<int64_t>(T) * rm.rs;
   const double* mb = m64 + static_cast<int64_t>(b) * D;
   const int vecs = D >> 3;
   for (int t0 = 0; t0 < nb; t0 += 4) {
@@ -401,7 +414,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
       uint4 q[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        q[u] = t0 + u < nb ? __ldg(reinterpret_cast<const uint4*>(Nb + static_cast<int64_t>(band_idx[t0 + u]) * D) + v)
+        q[u] = t0 + u < nb ? __ldg(reinterpret_cast<const uint4*>(Nb + static_cast<int64_t>(band_idx[t0 + u]) * rm.rs) + v)
                            : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -482,9 +495,14 @@ select_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, 
 
 }  // namespace
 
-wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int batch, int32_t* keep_idx,
+wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int chunks, int32_t* keep_idx,
                           float* scores_out, cudaStream_t s) {
-  const int T = ctx->cfg.tokens_per_frame, D = ctx->D, NA = ctx->NA, n_keep = ctx->cfg.n_keep;
+  const int T = ctx->cfg.tokens_per_frame, NA = ctx->NA, n_keep = ctx->cfg.n_keep;
+  // whole-token keys: one problem per chunk, D columns; per-head keys: n_heads problems per chunk, 128 columns each
+  const bool per_head = ctx->cfg.score_mode == WK_SCORE_PER_HEAD;
+  const int D = per_head ? kHeadDim : ctx->D;
+  const int batch = per_head ? chunks * ctx->cfg.n_heads : chunks;
+  const RowMap rm{stride, ctx->D, per_head ? ctx->cfg.n_heads : 1};
   uint8_t* sc = ctx->scratch_base;
   float* m32 = reinterpret_cast<float*>(sc + ctx->sl.m32_off);
   double* m64 = reinterpret_cast<double*>(sc + ctx->sl.m64_off);
@@ -502,11 +520,11 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       n_norm_parts = (D + 511) / 512;
       double* inv_norm = reinterpret_cast<double*>(sc + ctx->sl.inv_off);
       const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), batch);
-      anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, D, inv_norm);
+      anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const int threads = ((D / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
       const dim3 grid_acc(parts * kColSplit, batch);
-      anchor_accumulate<<<grid_acc, threads, 0, s>>>(K, stride, T, D, parts, inv_norm, partial);
+      anchor_accumulate<<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const dim3 grid_r((D + 511) / 512, batch);
       anchor_reduce<<<grid_r, 256, 0, s>>>(partial, T, D, parts, m64, m32, mnorm);
@@ -520,7 +538,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
     const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, batch);
-    score_pass<<<grid_s, kScoreThreads, static_cast<size_t>(D) * sizeof(float), s>>>(K, stride, T, NA, D, m32, s32,
+    score_pass<<<grid_s, kScoreThreads, static_cast<size_t>(D) * sizeof(float), s>>>(K, rm, T, NA, D, m32, s32,
                                                                                     scores_out, ctx->status_dev);
     if ((st = after_launch(ctx)) != WK_OK) return st;
   }
@@ -529,7 +547,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   if (smem_sel > 48 * 1024)
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(smem_sel)));
-  select_pass<<<batch, kSelectThreads, smem_sel, s>>>(K, stride, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts, keep_idx,
+  select_pass<<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts, keep_idx,
                                                      ctx->status_dev);
   return after_launch(ctx);
 }

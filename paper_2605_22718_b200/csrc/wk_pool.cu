@@ -7,26 +7,28 @@ namespace {
 
 constexpr int kAppendThreads = 256;
 
-// grid = (ceil(C / rows_per_cta), n_layers_in_call, 2 [K|V]); one warp per kept row, 16-byte vectors.
+// grid = (ceil(C / rows_per_cta), n_layers_in_call, 2 [K|V]); one warp per kept row, 16-byte vectors.  With per-head
+// keep-sets (hs = n_heads index lists per layer) every 128-column block of a stored row has its own source token.
 __global__ void __launch_bounds__(kAppendThreads)
 append_rows(const __nv_bfloat16* __restrict__ Ksrc, const __nv_bfloat16* __restrict__ Vsrc, int64_t stride,
-            const int32_t* __restrict__ keep_idx, int C, int FT, int D, __nv_bfloat16* __restrict__ Kdst,
+            const int32_t* __restrict__ keep_idx, int hs, int C, int FT, int D, __nv_bfloat16* __restrict__ Kdst,
             __nv_bfloat16* __restrict__ Vdst, int64_t dst_layer_stride, int rows_per_cta, uint32_t* __restrict__ status) {
   const int l = blockIdx.y, which = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const __nv_bfloat16* src = (which ? Vsrc : Ksrc) + static_cast<int64_t>(l) * stride;
   __nv_bfloat16* dst = (which ? Vdst : Kdst) + static_cast<int64_t>(l) * dst_layer_stride;
-  const int32_t* idx = keep_idx + static_cast<int64_t>(l) * C;
-  const int vecs = D >> 3;
+  const int32_t* idx = keep_idx + static_cast<int64_t>(l) * hs * C;
+  const int vecs = D >> 3, vecs_per_list = vecs / hs;
   const int r0 = blockIdx.x * rows_per_cta, r1 = min(C, r0 + rows_per_cta);
   for (int r = r0 + warp; r < r1; r += kAppendThreads / 32) {
-    const int j = idx[r];
-    if (j < 0 || j >= FT) {                       // never dereference a bad index
-      if (lane == 0) atomicOr(status, WK_DEV_BAD_SLOT);
-      continue;
-    }
-    const uint4* s = reinterpret_cast<const uint4*>(src + static_cast<int64_t>(j) * D);
     uint4* d = reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * D);
-    for (int v = lane; v < vecs; v += 32) d[v] = __ldg(s + v);
+    for (int v = lane; v < vecs; v += 32) {
+      const int j = idx[(v / vecs_per_list) * C + r];
+      if (j < 0 || j >= FT) {                     // never dereference a bad index
+        atomicOr(status, WK_DEV_BAD_SLOT);
+        continue;
+      }
+      d[v] = __ldg(reinterpret_cast<const uint4*>(src + static_cast<int64_t>(j) * D) + v);
+    }
   }
 }
 
@@ -48,7 +50,8 @@ wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfl
   __nv_bfloat16* Vdst = ctx->Vpool + layer0 * layer_stride + slot * slot_elems;
   const int rows_per_cta = 32;
   const dim3 grid((C + rows_per_cta - 1) / rows_per_cta, n, 2);
-  append_rows<<<grid, kAppendThreads, 0, s>>>(K, V, stride, keep_idx, C, ctx->FT, D, Kdst, Vdst, layer_stride,
+  const int hs = ctx->cfg.score_mode == WK_SCORE_PER_HEAD ? ctx->cfg.n_heads : 1;
+  append_rows<<<grid, kAppendThreads, 0, s>>>(K, V, stride, keep_idx, hs, C, ctx->FT, D, Kdst, Vdst, layer_stride,
                                               rows_per_cta, ctx->status_dev);
   return after_launch(ctx);
 }

@@ -34,8 +34,8 @@ class Scenario:
     """A pool filled through wk_compress_chunk + wk_pool_append, mirrored in the oracle's PoolModel."""
 
     def __init__(self, kv, seed: int, sigma: float, n_layers: int, T: int, H: int, n_keep: int, pool_slots: int,
-                 F: int = 3):
-        self.kv, self.seed, self.sigma = kv, seed, sigma
+                 F: int = 3, per_head: bool = False):
+        self.kv, self.seed, self.sigma, self.per_head = kv, seed, sigma, per_head
         self.L, self.T, self.H, self.D, self.F, self.n_keep = n_layers, T, H, H * 128, F, n_keep
         self.pool = o.PoolModel(n_slots=pool_slots, n_layers=n_layers)
         self.margins = []
@@ -52,7 +52,10 @@ class Scenario:
         keep = self.kv.compress_chunk(Kd)
         ref = []
         for l in range(self.L):
-            idx, _, margin = o.compress_chunk(K[l], self.T, self.n_keep)
+            if self.per_head:
+                idx, _, margin = o.compress_chunk_per_head(K[l], self.T, self.n_keep, self.H)
+            else:
+                idx, _, margin = o.compress_chunk(K[l], self.T, self.n_keep)
             ref.append(idx)
             self.margins.append(margin)
         if check:
