@@ -48,13 +48,18 @@ __device__ __forceinline__ float warp_sum(float v) {
 // Where the rows of problem b live.  A chunk is [F*T][rs] bf16; with whole-token keys (one keep-set per chunk) a
 // problem is a chunk and D = rs; with per-head keys a chunk holds hs = n_heads problems, problem (chunk, h) owning
 // columns [h*D, (h+1)*D) of every row, D = head_dim.
+// The kernels are instantiated for both cases, so that the whole-key case keeps its plain arithmetic (row pitch = D).
 struct RowMap {
   int64_t stride;   // elements between chunks
   int rs;           // elements between token rows
   int hs;           // problems per chunk
+  template <bool kPerHead>
   __device__ __forceinline__ const __nv_bfloat16* base(const __nv_bfloat16* K, int b, int D) const {
-    return K + static_cast<int64_t>(b / hs) * stride + static_cast<int64_t>(b % hs) * D;
+    if (kPerHead) return K + static_cast<int64_t>(b / hs) * stride + static_cast<int64_t>(b % hs) * D;
+    return K + static_cast<int64_t>(b) * stride;
   }
+  template <bool kPerHead>
+  __device__ __forceinline__ int pitch(int D) const { return kPerHead ? rs : D; }
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -64,13 +69,15 @@ struct RowMap {
 //                      a_i[8t..] / |a_i| over the rows of its slice in fp64; the anchor rows come from L2 the second
 //                      time.  The last CTA of a problem adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|.
 // ------------------------------------------------------------------------------------------------
+template <bool kPerHead>
 __global__ void __launch_bounds__(kAnchorThreads)
 anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, double* __restrict__ inv_norm) {
   const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
   if (r >= T) return;
   const int vecs = D >> 3;
-  const uint4* row = reinterpret_cast<const uint4*>(rm.base(K, b, D) + static_cast<int64_t>(r) * rm.rs);
+  const uint4* row =
+      reinterpret_cast<const uint4*>(rm.base<kPerHead>(K, b, D) + static_cast<int64_t>(r) * rm.pitch<kPerHead>(D));
   double n2a = 0.0, n2b = 0.0;
   for (int v0 = lane; v0 < vecs; v0 += 128) {
     uint4 q[4];
@@ -91,6 +98,7 @@ anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, doubl
   if (lane == 0) inv_norm[static_cast<int64_t>(b) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
 }
 
+template <bool kPerHead>
 __global__ void __launch_bounds__(512)
 anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, int parts,
                   const double* __restrict__ inv_norm, double* __restrict__ partial) {
@@ -98,8 +106,8 @@ anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, 
   const int tid = threadIdx.x, nthreads = blockDim.x;
   const int vecs = D >> 3;
   const int vec = csplit * nthreads + tid;   // the 16-byte column group this thread owns
-  const uint4* Kb = reinterpret_cast<const uint4*>(rm.base(K, b, D));
-  const int64_t rsv = rm.rs >> 3;   // row pitch in 16-byte vectors
+  const uint4* Kb = reinterpret_cast<const uint4*>(rm.base<kPerHead>(K, b, D));
+  const int rsv = rm.pitch<kPerHead>(D) >> 3;   // row pitch in 16-byte vectors
   const double* inv = inv_norm + static_cast<int64_t>(b) * T;
   if (vec < vecs) {
     double acc[8];
@@ -237,6 +245,7 @@ anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int
 // Per lane the fp32 accumulation is a chain of 8 * ceil(D/256) fused multiply-adds followed by five
 // shuffle additions; select_pass derives its error band from exactly this order.
 // ------------------------------------------------------------------------------------------------
+template <bool kPerHead>
 __global__ void __launch_bounds__(kScoreThreads)
 score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
            const float* __restrict__ m32, float* __restrict__ s32, float* __restrict__ scores_out,
@@ -250,14 +259,15 @@ score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
   const int vecs = D >> 3;
   const int j0 = blockIdx.x * kScoreRowsPerCta;
   const int j1 = min(NA, j0 + kScoreRowsPerCta);
-  const __nv_bfloat16* Kb = rm.base(K, b, D) + static_cast<int64_t>(T) * rm.rs;
+  const int pitch = rm.pitch<kPerHead>(D);
+  const __nv_bfloat16* Kb = rm.base<kPerHead>(K, b, D) + static_cast<int64_t>(T) * pitch;
   // two rows per warp at a time, so that twice as many 16-byte loads are in flight
   constexpr int W = kScoreThreads / 32;
   for (int j = j0 + warp; j < j1; j += 2 * W) {
     const int jb = j + W;
     const bool has_b = jb < j1;
-    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * rm.rs);
-    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * rm.rs);
+    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * pitch);
+    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * pitch);
     float dot_a = 0.f, n2_a = 0.f, dot_b = 0.f, n2_b = 0.f;
     for (int v0 = lane; v0 < vecs; v0 += 128) {
       uint4 qa[4], qb[4];
@@ -311,6 +321,7 @@ __device__ __forceinline__ float key_f32(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
+template <bool kPerHead>
 __global__ void __launch_bounds__(kSelectThreads)
 select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D, int n_keep,
             const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
@@ -398,7 +409,8 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   const int need = n_keep - static_cast<int>(n_below);   // >= 1: the threshold token itself is in the band
   // exact fp64 scores of the band tokens: the whole CTA works on four tokens at a time (thread = one 16-byte vector
   // of the row), partial sums meet in shared memory and are added in a fixed order
-  const __nv_bfloat16* Nb = rm.base(K, b, D) + static_cast<int64_t>(T) * rm.rs;
+  const int pitch = rm.pitch<kPerHead>(D);
+  const __nv_bfloat16* Nb = rm.base<kPerHead>(K, b, D) + static_cast<int64_t>(T) * pitch;
   const double* mb = m64 + static_cast<int64_t>(b) * D;
   const int vecs = D >> 3;
   for (int t0 = 0; t0 < nb; t0 += 4) {
@@ -414,7 +426,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
       uint4 q[4];
 #pragma unroll
       for (int u = 0; u < 4; ++u)
-        q[u] = t0 + u < nb ? __ldg(reinterpret_cast<const uint4*>(Nb + static_cast<int64_t>(band_idx[t0 + u]) * rm.rs) + v)
+        q[u] = t0 + u < nb ? __ldg(reinterpret_cast<const uint4*>(Nb + static_cast<int64_t>(band_idx[t0 + u]) * pitch) + v)
                            : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
@@ -520,11 +532,13 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       n_norm_parts = (D + 511) / 512;
       double* inv_norm = reinterpret_cast<double*>(sc + ctx->sl.inv_off);
       const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), batch);
-      anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
+      if (per_head) anchor_norms<true><<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
+      else anchor_norms<false><<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const int threads = ((D / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
       const dim3 grid_acc(parts * kColSplit, batch);
-      anchor_accumulate<<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
+      if (per_head) anchor_accumulate<true><<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
+      else anchor_accumulate<false><<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const dim3 grid_r((D + 511) / 512, batch);
       anchor_reduce<<<grid_r, 256, 0, s>>>(partial, T, D, parts, m64, m32, mnorm);
@@ -538,17 +552,27 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
     const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, batch);
-    score_pass<<<grid_s, kScoreThreads, static_cast<size_t>(D) * sizeof(float), s>>>(K, rm, T, NA, D, m32, s32,
-                                                                                    scores_out, ctx->status_dev);
+    const size_t smem_m = static_cast<size_t>(D) * sizeof(float);
+    if (per_head)
+      score_pass<true><<<grid_s, kScoreThreads, smem_m, s>>>(K, rm, T, NA, D, m32, s32, scores_out, ctx->status_dev);
+    else
+      score_pass<false><<<grid_s, kScoreThreads, smem_m, s>>>(K, rm, T, NA, D, m32, s32, scores_out, ctx->status_dev);
     if ((st = after_launch(ctx)) != WK_OK) return st;
   }
   const size_t smem_sel = static_cast<size_t>(NA) * (4 + 4 + 8 + 1) + 16;
   if (smem_sel > 200 * 1024) return WK_ERR_SHAPE;
-  if (smem_sel > 48 * 1024)
-    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (smem_sel > 48 * 1024) {
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(smem_sel)));
-  select_pass<<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts, keep_idx,
-                                                     ctx->status_dev);
+    WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(smem_sel)));
+  }
+  if (per_head)
+    select_pass<true><<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts,
+                                                              keep_idx, ctx->status_dev);
+  else
+    select_pass<false><<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts,
+                                                               keep_idx, ctx->status_dev);
   return after_launch(ctx);
 }
 
