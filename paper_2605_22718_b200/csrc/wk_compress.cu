@@ -45,6 +45,9 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// The five kernels of one call depend on each other in a chain and are launched with launch_chained (wk_internal.cuh):
+// nothing is read or written before dep_wait(), so only launch latency and block scheduling overlap.
+
 // Where the rows of problem b live.  A chunk is [F*T][rs] bf16; with whole-token keys (one keep-set per chunk) a
 // problem is a chunk and D = rs; with per-head keys a chunk holds hs = n_heads problems, problem (chunk, h) owning
 // columns [h*D, (h+1)*D) of every row, D = head_dim.
@@ -72,6 +75,7 @@ struct RowMap {
 template <bool kPerHead>
 __global__ void __launch_bounds__(kAnchorThreads)
 anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, double* __restrict__ inv_norm) {
+  dep_release();
   const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
   if (r >= T) return;
@@ -102,6 +106,8 @@ template <bool kPerHead>
 __global__ void __launch_bounds__(512)
 anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, int parts,
                   const double* __restrict__ inv_norm, double* __restrict__ partial) {
+  dep_wait();
+  dep_release();
   const int b = blockIdx.y, part = blockIdx.x / kColSplit, csplit = blockIdx.x % kColSplit;
   const int tid = threadIdx.x, nthreads = blockDim.x;
   const int vecs = D >> 3;
@@ -145,6 +151,8 @@ __global__ void __launch_bounds__(256)
 anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, double* __restrict__ m64, float* __restrict__ m32,
               double* __restrict__ mnorm2_part) {
   __shared__ double red2[8];
+  dep_wait();
+  dep_release();
   const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int c = 2 * (blockIdx.x * 256 + tid);
   const double* pb = partial + static_cast<int64_t>(b) * parts * D;
@@ -251,6 +259,8 @@ score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
            const float* __restrict__ m32, float* __restrict__ s32, float* __restrict__ scores_out,
            uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
+  dep_release();
   float4* m = reinterpret_cast<float4*>(smem);   // [D/4]
   const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
@@ -327,6 +337,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
             const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
             int n_norm_parts, int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem);                       // [NA]
   int32_t* band_idx = reinterpret_cast<int32_t*>(keys + NA);                // [NA]
   double* band_s = reinterpret_cast<double*>(band_idx + NA);                // [NA] (8-byte aligned: 8*NA)
@@ -537,11 +548,11 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const int threads = ((D / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
       const dim3 grid_acc(parts * kColSplit, batch);
-      if (per_head) anchor_accumulate<true><<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
-      else anchor_accumulate<false><<<grid_acc, threads, 0, s>>>(K, rm, T, D, parts, inv_norm, partial);
+      if (per_head) launch_chained(anchor_accumulate<true>, grid_acc, dim3(threads), 0, s, K, rm, T, D, parts, inv_norm, partial);
+      else launch_chained(anchor_accumulate<false>, grid_acc, dim3(threads), 0, s, K, rm, T, D, parts, inv_norm, partial);
       if ((st = after_launch(ctx)) != WK_OK) return st;
       const dim3 grid_r((D + 511) / 512, batch);
-      anchor_reduce<<<grid_r, 256, 0, s>>>(partial, T, D, parts, m64, m32, mnorm);
+      launch_chained(anchor_reduce, grid_r, dim3(256), 0, s, partial, T, D, parts, m64, m32, mnorm);
     } else {
       const size_t smem_acc = static_cast<size_t>(D) * sizeof(double);
       if (smem_acc > 200 * 1024) return WK_ERR_SHAPE;
@@ -554,9 +565,11 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
     const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, batch);
     const size_t smem_m = static_cast<size_t>(D) * sizeof(float);
     if (per_head)
-      score_pass<true><<<grid_s, kScoreThreads, smem_m, s>>>(K, rm, T, NA, D, m32, s32, scores_out, ctx->status_dev);
+      launch_chained(score_pass<true>, grid_s, dim3(kScoreThreads), smem_m, s, K, rm, T, NA, D, m32, s32, scores_out,
+                     ctx->status_dev);
     else
-      score_pass<false><<<grid_s, kScoreThreads, smem_m, s>>>(K, rm, T, NA, D, m32, s32, scores_out, ctx->status_dev);
+      launch_chained(score_pass<false>, grid_s, dim3(kScoreThreads), smem_m, s, K, rm, T, NA, D, m32, s32, scores_out,
+                     ctx->status_dev);
     if ((st = after_launch(ctx)) != WK_OK) return st;
   }
   const size_t smem_sel = static_cast<size_t>(NA) * (4 + 4 + 8 + 1) + 16;
@@ -568,11 +581,11 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
                                           static_cast<int>(smem_sel)));
   }
   if (per_head)
-    select_pass<true><<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts,
-                                                              keep_idx, ctx->status_dev);
+    launch_chained(select_pass<true>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
+                   n_norm_parts, keep_idx, ctx->status_dev);
   else
-    select_pass<false><<<batch, kSelectThreads, smem_sel, s>>>(K, rm, T, NA, D, n_keep, s32, m64, mnorm, n_norm_parts,
-                                                               keep_idx, ctx->status_dev);
+    launch_chained(select_pass<false>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
+                   n_norm_parts, keep_idx, ctx->status_dev);
   return after_launch(ctx);
 }
 

@@ -118,6 +118,29 @@ wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfl
                         int64_t stride, const int32_t* keep_idx, cudaStream_t s);
 wk_status launch_slot_mark(wk_ctx* ctx, int slot, int valid, const float* pose, cudaStream_t s);
 wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out, cudaStream_t s);
+// Kernels of one call that depend on each other in a chain are launched so that a kernel may be scheduled while its
+// predecessor drains (programmatic dependent launch): dep_wait() at the top of a kernel returns once the predecessor
+// has completed and its writes are visible; dep_release() lets the successor's launch proceed.  A kernel launched the
+// ordinary way after a chained one still waits for its full completion.
+#ifdef __CUDACC__
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+inline void launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // errors surface in after_launch
+}
+#endif
+
 size_t retrieve_scan_scratch_bytes();
 wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* valid, int64_t n, const float* cur_pose,
                                int k, int32_t* ids_out, double* dist_out, int out_capacity, void* scratch, cudaStream_t s);

@@ -59,6 +59,7 @@ __device__ __forceinline__ Cand candidate(const float4 a, const float4 b, const 
 struct Cur8 { float v[8]; };
 
 __global__ void scan_init(ScanHeader* h) {
+  dep_release();
   h->t_max_bits = 0ull;
   h->dot_min_bits = static_cast<unsigned long long>(__double_as_longlong(2.0));
   h->n_valid = 0ull;
@@ -67,6 +68,8 @@ __global__ void scan_init(ScanHeader* h) {
 
 __global__ void __launch_bounds__(kScanThreads)
 scan_max(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, Cur8 cur, ScanHeader* h) {
+  dep_wait();
+  dep_release();
   double mt = 0.0, mdot = 2.0;
   unsigned int cnt = 0;
   for (int64_t i = static_cast<int64_t>(blockIdx.x) * kScanThreads + threadIdx.x; i < n;
@@ -153,6 +156,8 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   __shared__ int s_cnt, s_npend[2];
   __shared__ double s_tau;
   __shared__ float s_tau_hi;
+  dep_wait();
+  dep_release();
   TopK top;
   top.init(s_key, s_i, &s_cnt, &s_tau, k);
   const double mt = __longlong_as_double(static_cast<long long>(h->t_max_bits));
@@ -190,7 +195,7 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   };
   if (threadIdx.x == 0) s_npend[0] = s_npend[1] = 0;
   refresh();
-  // Round 0 takes kScanWarm candidates and cuts the list at once: that gives a first k-th best, after which few of
+  // The first pass over kScanWarm candidates cuts the list at once: that gives a first k-th best, after which few of
   // the later candidates pass the bound.  Later rounds take kScanUnroll candidates per thread.
   const int64_t warm0 = static_cast<int64_t>(blockIdx.x) * kScanWarm;
   const int64_t warm_all = static_cast<int64_t>(gridDim.x) * kScanWarm;
@@ -257,6 +262,7 @@ scan_merge(const ScanEntry* __restrict__ block_out, int n_lists, int k, int out_
   __shared__ int32_t s_widx[kMergeThreads / 32];
   __shared__ int s_wlist[kMergeThreads / 32];
   __shared__ int s_winner;
+  dep_wait();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned long long kInf = static_cast<unsigned long long>(__double_as_longlong(INFINITY));
   int pos = 0;   // head of this thread's list; the entry after it is fetched ahead, off the critical path
@@ -347,11 +353,13 @@ wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* v
   scan_init<<<1, 1, 0, s>>>(h);
   if ((st = after_launch(ctx)) != WK_OK) return st;
   const float4* p4 = reinterpret_cast<const float4*>(poses);
-  scan_max<<<static_cast<unsigned>(blocks), kScanThreads, 0, s>>>(p4, valid, n, cur, h);
+  launch_chained(scan_max, dim3(static_cast<unsigned>(blocks)), dim3(kScanThreads), 0, s, p4, valid, n, cur, h);
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  scan_select<<<static_cast<unsigned>(sel_blocks), kSelThreads, 0, s>>>(p4, valid, n, cur, h, k, block_out);
+  launch_chained(scan_select, dim3(static_cast<unsigned>(sel_blocks)), dim3(kSelThreads), 0, s, p4, valid, n, cur, h, k,
+                 block_out);
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  scan_merge<<<1, kMergeThreads, 0, s>>>(block_out, static_cast<int>(sel_blocks), k, out_capacity, ids_out, dist_out);
+  launch_chained(scan_merge, dim3(1), dim3(kMergeThreads), 0, s, block_out, static_cast<int>(sel_blocks), k, out_capacity,
+                 ids_out, dist_out);
   return after_launch(ctx);
 }
 
