@@ -12,29 +12,36 @@ What each function follows
 * ``compression_scores_factorised``   -- the same quantity after pulling the sum over anchors
   inside the dot product: s_j = (k_j / |k_j|) . m with m = (1/T) sum_i a_i / |a_i|.  An exact
   algebraic identity; both forms are kept and compared.
-* ``keep_set`` -- Section 4.3, "pool these scores across all non-anchor frames and retain the
-  bottom P %": the n_keep lowest pooled scores; the compressed chunk is every anchor token
-  plus those.
+* ``keep_set`` -- Section 4.3: the scores of all non-anchor frames go into one pool and the
+  lowest-scoring share of it is retained: the n_keep lowest pooled scores; the compressed chunk
+  is every anchor token plus those.
+* ``compress_chunk_per_head`` -- the same, with one attention head's key as the vector of Eq. 5
+  (the other reading of R1): one keep-set per head.
 * ``retrieval_distances`` / ``retrieve`` -- Eq. 4 (Section 4.2) with the distance of Section 5.1:
   squared-L2 translation distance and geodesic rotation distance, each normalised across
   the candidate set, summed; the smallest k win.
 * ``attention`` -- the attention of Section 4.2's assembled window: every query attends,
   unmasked, to [dense segments ..., retrieved pool chunks ...]; softmax(scale q K^T) V.
-* ``PoolModel`` -- the chunk pool of Section 4.2 ("stored ... rather than discarded, each
-  indexed by" its pose) as a slot table.
+* ``PoolModel`` -- the chunk pool of Section 4.2 (evicted chunks are kept, each filed under its
+  camera pose) as a slot table.
+* ``query_scores`` / ``retrieve_query`` -- the query-based retrieval of Appendix C: a stored chunk's
+  score is the softmax mass the current queries put on its keys (reading R12 below).
 
 Readings taken where the paper is silent (each is one line of code below)
 -------------------------------------------------------------------------
 R1  d in Eq. 5 is the whole per-layer key of a token (all heads concatenated); one keep-set
-    per (layer, chunk).
-R2  "bottom P %" is passed as the integer n_keep; ties are broken by the lowest pooled index.
+    per (layer, chunk).  The per-head reading (d = head_dim, one keep-set per head) is kept beside it.
+R2  the retained share of the pool is passed as the integer n_keep; ties are broken by the lowest pooled index.
 R3  a zero key has cosine 0 with everything (and still counts in the 1/T).
-R4  "normalised across the candidate set" = divided by the maximum over the candidates; a
+R4  normalising a distance term over the candidates = dividing it by its maximum over them; a
     term whose maximum is 0 contributes 0.
 R5  geodesic rotation distance = 2 acos(min(1, |<q_cur, q_i>|)), in [0, pi].
 R6  retrieval ties are broken by the lowest slot index; k > M returns all M.
 R7  softmax scale = 1 / sqrt(head_dim); no mask, no positional re-encoding of stored keys.
 R8  a retrieved slot listed twice is attended twice (multiset semantics).
+R12 query-based retrieval: one layer's queries, logits scaled by 1/sqrt(head_dim), softmax over all
+    stored keys of that layer per head and query row, a chunk's mass = the sum over its keys,
+    score = the mean over heads and rows; ties to the lowest slot.
 
 Pins: see tests/test_oracle_*.py (closed forms, brute force on tiny inputs, invariants, and
 independent textbook/library restatements).  No function here is "parity unpinned".
