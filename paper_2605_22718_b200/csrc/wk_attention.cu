@@ -365,8 +365,10 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       }
     }
   } else if (warp == kMmaWarp) {
-    // ------------------------------------------------------------------ MMA issue (one thread)
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issue
+    // The whole warp runs the control flow (waits, counters, descriptor arithmetic) so that everything stays
+    // warp-uniform; one elected lane issues the tensor-core instructions and the commits.
+    {
       const uint32_t idesc_qk = idesc_bf16_f32(128, 128, 0, 0);
       const uint32_t idesc_pv = idesc_bf16_f32(128, 128, 0, 1);
       const uint32_t aQ = smem_u32(sQ), aK = smem_u32(sK), aV = smem_u32(sV);
@@ -374,28 +376,41 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       const uint32_t hi = smem_desc_hi_sw128(1024);
       const uint32_t q_lo0 = smem_desc_lo(aQ, 16), q_lo1 = smem_desc_lo(aQ + kTileBytes, 16);
       const uint32_t k_lo0 = smem_desc_lo(aK, 16), v_lo0 = smem_desc_lo(aV, kHalfTileBytes);
-      auto issue_s = [&](int i, int st) {
+      auto issue_s = [&](int i, uint32_t st) {
         const uint32_t d = tmem + i * 128;
         const uint32_t a_lo = i ? q_lo1 : q_lo0, b_lo = k_lo0 + st * (kTileBytes >> 4);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const uint32_t off = (k >> 2) * (kHalfTileBytes >> 4) + (k & 3) * 2;   // 32 bytes per step inside a 128-byte row
-          mma_ss_lohi(d, a_lo + off, b_lo + off, hi, idesc_qk, k > 0);
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t off = (k >> 2) * (kHalfTileBytes >> 4) + (k & 3) * 2;   // 32 bytes per step inside a 128-byte row
+            mma_ss_lohi(d, a_lo + off, b_lo + off, hi, idesc_qk, k > 0);
+          }
         }
+        __syncwarp();
       };
-      auto issue_pv = [&](int i, int st, bool accumulate) {
+      auto issue_pv = [&](int i, uint32_t st, bool accumulate) {
         const uint32_t d = tmem + 256 + i * 128;
         const uint32_t b_lo = v_lo0 + st * (kTileBytes >> 4);
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          // A = P from tensor memory (bf16 pairs, 8 columns per K = 16 step); B = V, rows = K dimension, MN-major:
-          // 16 rows of 128 bytes = 2048 bytes per step
-          mma_ts_lohi(d, tmem + i * 128 + k * 8, b_lo + k * 128, hi, idesc_pv, (accumulate || k > 0) ? 1u : 0u);
+          for (int k = 0; k < 8; ++k) {
+            // A = P from tensor memory (bf16 pairs, 8 columns per K = 16 step); B = V, rows = K dimension, MN-major:
+            // 16 rows of 128 bytes = 2048 bytes per step
+            mma_ts_lohi(d, tmem + i * 128 + k * 8, b_lo + k * 128, hi, idesc_pv, (accumulate || k > 0) ? 1u : 0u);
+          }
         }
+        __syncwarp();
+      };
+      auto commit = [&](uint64_t* bar) {
+        if (elect_one()) mma_commit(bar);
+        __syncwarp();
       };
       PieceWalker walk;
       walk.init(p);
       Piece pc;
+      // stage and phase of the K tile whose Q K^T is issued next / of the V tile whose P V is issued next: counters
+      // instead of divisions on the issuing path
+      uint32_t ks = 0, kph = 0, vs = 0, vph = 0;
       uint32_t g0 = 0, g1 = 0, n = 0;   // running tile counts of the two Q tiles, running piece count
       uint32_t e0 = 0, e1 = 0;          // pieces in which Q tile 0 / 1 produced output so far
       WK_PROF_DECL
@@ -412,7 +427,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
         if (!(ok = wait_or_abort(&bars.q_full, n & 1, &s_abort, p.status))) break;
         ++n;
         if (n_eff == 0) {
-          mbar_arrive(&bars.q_empty);
+          if (lane == 0) mbar_arrive(&bars.q_empty);
           continue;
         }
         // O0 / O1 are about to be overwritten: the epilogue of the last piece that used them must have read them.
@@ -424,50 +439,51 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           if (e1 > 0 && !(ok = wait_or_abort(&bars.o_free[1], (e1 - 1) & 1, &s_abort, p.status))) break;
           ++e1;
         }
+        auto next_k = [&]() { if (++ks == kStagesK) { ks = 0; kph ^= 1; } };
+        auto next_v = [&]() { if (++vs == kStagesV) { vs = 0; vph ^= 1; } };
         {
-          const int st = g0 % kStagesK;
-          if (!(ok = wait_or_abort(&bars.k_full[st], (g0 / kStagesK) & 1, &s_abort, p.status))) break;
+          if (!(ok = wait_or_abort(&bars.k_full[ks], kph, &s_abort, p.status))) break;
           tc_fence_after();
-          issue_s(0, st);
-          mma_commit(&bars.s_full[0]);
-          if (q1) { issue_s(1, st); mma_commit(&bars.s_full[1]); }
-          mma_commit(&bars.k_empty[st]);
-          if (n_eff == 1) mma_commit(&bars.q_empty);
+          issue_s(0, ks);
+          commit(&bars.s_full[0]);
+          if (q1) { issue_s(1, ks); commit(&bars.s_full[1]); }
+          commit(&bars.k_empty[ks]);
+          if (n_eff == 1) commit(&bars.q_empty);
+          next_k();
         }
         for (int j = 0; j < n_eff; ++j) {
-          const uint32_t g = g0 + j;
-          const int st = g % kStagesV, stn = (g + 1) % kStagesK;   // V stage of this tile, K stage of the next
-          const uint32_t ph = (g / kStagesV) & 1, phn = ((g + 1) / kStagesK) & 1;
           const bool more = j + 1 < n_eff;
           WK_PROF(10, blockIdx.x == 0);
-          if (!kLse && !(ok = wait_or_abort(&bars.v_full[st], ph, &s_abort, p.status))) break;
+          if (!kLse && !(ok = wait_or_abort(&bars.v_full[vs], vph, &s_abort, p.status))) break;
           WK_PROF(11, blockIdx.x == 0);
-          if (!(ok = wait_or_abort(&bars.p_full[0], g & 1, &s_abort, p.status))) break;
+          if (!(ok = wait_or_abort(&bars.p_full[0], (g0 + j) & 1, &s_abort, p.status))) break;
           WK_PROF(12, blockIdx.x == 0);
           tc_fence_after();
-          if (!kLse) issue_pv(0, st, j > 0);
-          mma_commit(&bars.o_done[0]);
+          if (!kLse) issue_pv(0, vs, j > 0);
+          commit(&bars.o_done[0]);
           if (more) {
             WK_PROF(13, blockIdx.x == 0);
-            if (!(ok = wait_or_abort(&bars.k_full[stn], phn, &s_abort, p.status))) break;
+            if (!(ok = wait_or_abort(&bars.k_full[ks], kph, &s_abort, p.status))) break;
             WK_PROF(14, blockIdx.x == 0);
             tc_fence_after();
-            issue_s(0, stn);
-            mma_commit(&bars.s_full[0]);
+            issue_s(0, ks);
+            commit(&bars.s_full[0]);
           }
           if (q1) {
             WK_PROF(15, blockIdx.x == 0);
             if (!(ok = wait_or_abort(&bars.p_full[1], (g1 + j) & 1, &s_abort, p.status))) break;
             WK_PROF(16, blockIdx.x == 0);
             tc_fence_after();
-            if (!kLse) issue_pv(1, st, j > 0);
-            mma_commit(&bars.o_done[1]);
+            if (!kLse) issue_pv(1, vs, j > 0);
+            commit(&bars.o_done[1]);
           }
-          if (!kLse) mma_commit(&bars.v_empty[st]);
+          if (!kLse) commit(&bars.v_empty[vs]);
+          next_v();
           if (more) {
-            if (q1) { issue_s(1, stn); mma_commit(&bars.s_full[1]); }
-            mma_commit(&bars.k_empty[stn]);
-            if (j + 2 == n_eff) mma_commit(&bars.q_empty);   // the last Q K^T of this piece has been issued
+            if (q1) { issue_s(1, ks); commit(&bars.s_full[1]); }
+            commit(&bars.k_empty[ks]);
+            if (j + 2 == n_eff) commit(&bars.q_empty);   // the last Q K^T of this piece has been issued
+            next_k();
           }
         }
         g0 += n_eff;
