@@ -32,9 +32,9 @@ METRIC = "memory-attn TFLOP/s over the whole chunk step (attention + retrieval +
 UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per memory_attention_kernel launch from the ncu capture summarised in
-# profiles/memory_attention_cfg2_shape.md (cfg2 per-call shape: 122.7 MB read + 5.5 MB written); it does not depend on
+# profiles/memory_attention_cfg2_shape.md (cfg2 per-call shape: 122.7 MB read + 5.4 MB written); it does not depend on
 # the pool size, so the small-pool capture stands for the full workload.  Other workloads report null.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 128.2e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 128.1e6
 
 
 def load_peaks():
