@@ -265,6 +265,30 @@ class ChunkStepBench:
         wk_compress_chunk over all layers of a chunk, and wk_retrieve."""
         torch, w, kv = self.torch, self.w, self.kv
         out = {}
+        # the attention call timed on its own: 5 warm-up calls, then 24 timed ones whose Q / O / window rotate over the
+        # layers' buffers (each call reads other memory than the one before it); median of per-call event times
+        pose = self.poses[w.pool_chunks % len(self.poses)]
+        _, n_sl = kv.retrieve(pose, w.k, slots_out=self.slots)
+
+        def attn_call(i):
+            l, s_ = i % w.n_layers, (i // w.n_layers) % w.denoise_steps
+            segs = [(self.curK[l], self.curV[l])]
+            if w.window_frames > 0:
+                rows = self.winK.shape[1] // w.window_segments
+                for q in range(w.window_segments):
+                    segs.append((self.winK[l, q * rows:(q + 1) * rows], self.winV[l, q * rows:(q + 1) * rows]))
+            kv.memory_attention(l, self.Q[l, s_], segs, self.slots, n_sl, O=self.O[l, s_], kv_splits=self.kv_splits)
+
+        for i in range(5):
+            attn_call(i)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(24)]
+        for i, (a, b) in enumerate(evs):
+            a.record()
+            attn_call(5 + i)
+            b.record()
+        torch.cuda.synchronize(self.dev)
+        us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
+        out["attention_isolated"] = {"us_per_call": us, "tflops": self.attention_flops_per_call() / us / 1e6, "calls": 24}
         for i in range(4):
             kv.compress_chunk(self.evK[i % len(self.evK)], keep_idx_out=self.keep)
         torch.cuda.synchronize(self.dev)
@@ -538,6 +562,8 @@ def run_ours(args, w: wi.Workload):
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if w.name.startswith("cfg2") else None,
                      "kernel": "memory_attention_kernel"},
+        "attention_isolated": dict(side["attention_isolated"],
+                                   frac_of_burst_peak=side["attention_isolated"]["tflops"] / peaks["bf16_tflops"]),
         "compress": side["compress"], "compress_per_head": side["compress_per_head"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
         "retrieve_scan": side["retrieve_scan"],
         "compress_append_bytes_per_step": comp_bytes,
