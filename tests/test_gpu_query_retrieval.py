@@ -109,3 +109,16 @@ def test_query_retrieval_cfg0_shape():
     # the query was not drawn from score within 0.5 % of each other: past rank 4 only validity is checked
     for k in (6, 12, 16):
         _check(kv, sc, 0, Qb, k)
+
+
+def test_query_retrieval_many_slots_matrix_game_heads():
+    """12 heads, 40 stored chunks of 1,320 tokens, 300 query rows (two q-pairs, the second without a second Q tile): the
+    launch shape of the benchmark's query-based retrieval (every slot a problem of its own, whole units per CTA)."""
+    w = wi.WORKLOADS["cfg1"]
+    kv, sc = _scene(T=w.T, H=w.n_heads, n_keep=w.n_keep, n_chunks=40, pool_slots=48, max_lq=300, seed=w.seed, n_layers=1)
+    kv.pool_evict(17)
+    sc.pool.evict(17)
+    Qb = _mixture_query(sc, 0, [(31, 120), (5, 80), (22, 60), (0, 40)])
+    assert Qb.shape[0] == 300
+    for k in (1, 2, 8):
+        _check(kv, sc, 0, Qb, k)

@@ -87,8 +87,8 @@ def test_scan_adversarial_order(kv):
     _check(kv, P[np.argsort(-d)].copy(), cur, 16)
 
 
-@pytest.mark.parametrize("log2n", [20, 24])
-def test_scan_full_size(kv, log2n):
+@pytest.mark.parametrize("log2n,k", [(20, 16), (20, 64), (24, 16)])
+def test_scan_full_size(kv, log2n, k):
     n = 1 << log2n
     poses = wi.random_poses(100 + log2n, n + 1)
-    _check(kv, poses[1:], poses[0], 16)
+    _check(kv, poses[1:], poses[0], k)
