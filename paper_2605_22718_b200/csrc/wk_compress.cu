@@ -72,16 +72,14 @@ struct RowMap {
 //                      a_i[8t..] / |a_i| over the rows of its slice in fp64; the anchor rows come from L2 the second
 //                      time.  The last CTA of a problem adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|.
 // ------------------------------------------------------------------------------------------------
-template <bool kPerHead>
 __global__ void __launch_bounds__(kAnchorThreads)
-anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, double* __restrict__ inv_norm) {
+anchor_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, double* __restrict__ inv_norm) {
   dep_release();
   const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
   if (r >= T) return;
   const int vecs = D >> 3;
-  const uint4* row =
-      reinterpret_cast<const uint4*>(rm.base<kPerHead>(K, b, D) + static_cast<int64_t>(r) * rm.pitch<kPerHead>(D));
+  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(r) * D);
   double n2a = 0.0, n2b = 0.0;
   for (int v0 = lane; v0 < vecs; v0 += 128) {
     uint4 q[4];
@@ -102,6 +100,50 @@ anchor_norms(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, doubl
   if (lane == 0) inv_norm[static_cast<int64_t>(b) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
 }
 
+// Per-head keys: the same pass over whole rows (all heads of a token are one contiguous row), with the sums taken per
+// 128-column block.  A warp covers 256 columns = two heads per step; lanes 0-15 reduce one head, lanes 16-31 the other.
+// Problem index of (chunk, head) = chunk * n_heads + head, as everywhere in the per-head path.
+__device__ __forceinline__ double half_warp_sum(double v) {
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float half_warp_sum(float v) {
+#pragma unroll
+  for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__global__ void __launch_bounds__(kAnchorThreads)
+head_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int H, double* __restrict__ inv_norm) {
+  dep_release();
+  const int chunk = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
+  if (r >= T) return;
+  const int vecs = D >> 3;
+  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(r) * D);
+  for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
+    uint4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+      double n2a = 0.0, n2b = 0.0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
+        n2a = fma(x0, x0, n2a);
+        n2b = fma(x1, x1, n2b);
+      }
+      const double n2 = half_warp_sum(n2a + n2b);
+      const int head = (v0 + 32 * u) >> 4;
+      if ((lane & 15) == 0 && head < H)
+        inv_norm[(static_cast<int64_t>(chunk) * H + head) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
+    }
+  }
+}
+
 template <bool kPerHead>
 __global__ void __launch_bounds__(512)
 anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, int parts,
@@ -112,9 +154,10 @@ anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, 
   const int tid = threadIdx.x, nthreads = blockDim.x;
   const int vecs = D >> 3;
   const int vec = csplit * nthreads + tid;   // the 16-byte column group this thread owns
-  const uint4* Kb = reinterpret_cast<const uint4*>(rm.base<kPerHead>(K, b, D));
-  const int rsv = rm.pitch<kPerHead>(D) >> 3;   // row pitch in 16-byte vectors
-  const double* inv = inv_norm + static_cast<int64_t>(b) * T;
+  // per-head keys: b is the chunk, the row is the whole token (D = all heads) and the norm is the one of this thread's head
+  const uint4* Kb = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * rm.stride);
+  const int rsv = D >> 3;   // row pitch in 16-byte vectors
+  const double* inv = inv_norm + (kPerHead ? (static_cast<int64_t>(b) * rm.hs + (vec >> 4)) : static_cast<int64_t>(b)) * T;
   if (vec < vecs) {
     double acc[8];
 #pragma unroll
@@ -147,9 +190,10 @@ anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, 
 
 // Adds the row slices of every problem in a fixed order: m64, m32 = fp32(m64) and this CTA's share of |m|^2.
 // grid = (ceil(D / 512), batch), 256 threads, two columns per thread; all loads are issued before the first addition.
+template <bool kPerHead>
 __global__ void __launch_bounds__(256)
-anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, double* __restrict__ m64, float* __restrict__ m32,
-              double* __restrict__ mnorm2_part) {
+anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, int H, double* __restrict__ m64,
+              float* __restrict__ m32, double* __restrict__ mnorm2_part) {
   __shared__ double red2[8];
   dep_wait();
   dep_release();
@@ -177,7 +221,12 @@ anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, doubl
   nn = warp_sum(nn);
   if (lane == 0) red2[warp] = nn;
   __syncthreads();
-  if (tid == 0) {
+  if (kPerHead) {
+    // a warp covers 64 columns: two warps per head, four heads per block; |m_h|^2 is one share per (chunk, head)
+    const int head = blockIdx.x * 4 + tid;
+    if (tid < 4 && head < H)
+      mnorm2_part[(static_cast<int64_t>(b) * H + head) * kMaxNormParts] = red2[2 * tid] + red2[2 * tid + 1];
+  } else if (tid == 0) {
     double t = 0.0;
     for (int w = 0; w < 8; ++w) t += red2[w];
     mnorm2_part[static_cast<int64_t>(b) * kMaxNormParts + blockIdx.x] = t;
@@ -253,9 +302,8 @@ anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int
 // Per lane the fp32 accumulation is a chain of 8 * ceil(D/256) fused multiply-adds followed by five
 // shuffle additions; select_pass derives its error band from exactly this order.
 // ------------------------------------------------------------------------------------------------
-template <bool kPerHead>
 __global__ void __launch_bounds__(kScoreThreads)
-score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
+score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D,
            const float* __restrict__ m32, float* __restrict__ s32, float* __restrict__ scores_out,
            uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
@@ -269,8 +317,8 @@ score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
   const int vecs = D >> 3;
   const int j0 = blockIdx.x * kScoreRowsPerCta;
   const int j1 = min(NA, j0 + kScoreRowsPerCta);
-  const int pitch = rm.pitch<kPerHead>(D);
-  const __nv_bfloat16* Kb = rm.base<kPerHead>(K, b, D) + static_cast<int64_t>(T) * pitch;
+  const int pitch = D;
+  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * pitch;
   // two rows per warp at a time, so that twice as many 16-byte loads are in flight
   constexpr int W = kScoreThreads / 32;
   for (int j = j0 + warp; j < j1; j += 2 * W) {
@@ -316,6 +364,61 @@ score_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D,
       if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
       s32[static_cast<int64_t>(b) * NA + jj] = sc;
       if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
+    }
+  }
+}
+
+// Per-head keys: whole rows again, the dot product and the squared norm taken per 128-column block (lanes 0-15 / 16-31
+// of a 256-column step).  Per lane and head: 8 fused multiply-adds, then 4 shuffle additions -- inside the error band
+// select_pass derives for D = 128.
+__global__ void __launch_bounds__(kScoreThreads)
+head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int H, const float* __restrict__ m32,
+           float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
+  dep_release();
+  float4* m = reinterpret_cast<float4*>(smem);   // [D/4]: the heads' mean unit anchors, side by side
+  const int chunk = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(chunk) * D);
+  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
+  __syncthreads();
+  const int vecs = D >> 3;
+  const int j0 = blockIdx.x * kScoreRowsPerCta;
+  const int j1 = min(NA, j0 + kScoreRowsPerCta);
+  const __nv_bfloat16* Kb = K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(T) * D;
+  constexpr int W = kScoreThreads / 32;
+  for (int j = j0 + warp; j < j1; j += W) {
+    const uint4* row = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
+    for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u;
+        float dot = 0.f, n2 = 0.f;
+        if (v < vecs) {
+          const float4 ma = m[2 * v], mb = m[2 * v + 1];
+          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x;
+            x = bf16lo(w[e]); dot = fmaf(x, mm[2 * e], dot); n2 = fmaf(x, x, n2);
+            x = bf16hi(w[e]); dot = fmaf(x, mm[2 * e + 1], dot); n2 = fmaf(x, x, n2);
+          }
+        }
+        dot = half_warp_sum(dot);
+        n2 = half_warp_sum(n2);
+        const int head = v >> 4;
+        if ((lane & 15) == 0 && head < H) {
+          const float sc = n2 > 0.f ? __fdiv_rn(dot, __fsqrt_rn(n2)) : 0.f;
+          if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + j;
+          s32[at] = sc;
+          if (scores_out) scores_out[at] = sc;
+        }
+      }
     }
   }
 }
@@ -521,11 +624,13 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
 wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int chunks, int32_t* keep_idx,
                           float* scores_out, cudaStream_t s) {
   const int T = ctx->cfg.tokens_per_frame, NA = ctx->NA, n_keep = ctx->cfg.n_keep;
-  // whole-token keys: one problem per chunk, D columns; per-head keys: n_heads problems per chunk, 128 columns each
+  // whole-token keys: one problem per chunk, D columns; per-head keys: n_heads problems per chunk, 128 columns each.
+  // The streaming kernels walk whole rows either way (DF columns); only the selection sees (chunk, head) problems.
   const bool per_head = ctx->cfg.score_mode == WK_SCORE_PER_HEAD;
-  const int D = per_head ? kHeadDim : ctx->D;
-  const int batch = per_head ? chunks * ctx->cfg.n_heads : chunks;
-  const RowMap rm{stride, ctx->D, per_head ? ctx->cfg.n_heads : 1};
+  const int H = ctx->cfg.n_heads, DF = ctx->D;
+  const int D = per_head ? kHeadDim : DF;
+  const int batch = per_head ? chunks * H : chunks;
+  const RowMap rm{stride, DF, per_head ? H : 1};
   uint8_t* sc = ctx->scratch_base;
   float* m32 = reinterpret_cast<float*>(sc + ctx->sl.m32_off);
   double* m64 = reinterpret_cast<double*>(sc + ctx->sl.m64_off);
@@ -538,37 +643,39 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   wk_status st = WK_OK;
   int n_norm_parts = 1;
   if (need_scores) {
-    const dim3 grid_a(parts, batch);
-    if (D <= 8192) {
-      n_norm_parts = (D + 511) / 512;
+    if (DF <= 8192) {
+      n_norm_parts = per_head ? 1 : (DF + 511) / 512;
       double* inv_norm = reinterpret_cast<double*>(sc + ctx->sl.inv_off);
-      const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), batch);
-      if (per_head) anchor_norms<true><<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
-      else anchor_norms<false><<<grid_n, kAnchorThreads, 0, s>>>(K, rm, T, D, inv_norm);
+      const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), chunks);
+      if (per_head) head_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, DF, H, inv_norm);
+      else anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, DF, inv_norm);
       if ((st = after_launch(ctx)) != WK_OK) return st;
-      const int threads = ((D / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
-      const dim3 grid_acc(parts * kColSplit, batch);
-      if (per_head) launch_chained(anchor_accumulate<true>, grid_acc, dim3(threads), 0, s, K, rm, T, D, parts, inv_norm, partial);
-      else launch_chained(anchor_accumulate<false>, grid_acc, dim3(threads), 0, s, K, rm, T, D, parts, inv_norm, partial);
+      const int threads = ((DF / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
+      const dim3 grid_acc(parts * kColSplit, chunks);
+      if (per_head) launch_chained(anchor_accumulate<true>, grid_acc, dim3(threads), 0, s, K, rm, T, DF, parts, inv_norm, partial);
+      else launch_chained(anchor_accumulate<false>, grid_acc, dim3(threads), 0, s, K, rm, T, DF, parts, inv_norm, partial);
       if ((st = after_launch(ctx)) != WK_OK) return st;
-      const dim3 grid_r((D + 511) / 512, batch);
-      launch_chained(anchor_reduce, grid_r, dim3(256), 0, s, partial, T, D, parts, m64, m32, mnorm);
+      const dim3 grid_r((DF + 511) / 512, chunks);
+      if (per_head) launch_chained(anchor_reduce<true>, grid_r, dim3(256), 0, s, partial, T, DF, parts, H, m64, m32, mnorm);
+      else launch_chained(anchor_reduce<false>, grid_r, dim3(256), 0, s, partial, T, DF, parts, H, m64, m32, mnorm);
     } else {
-      const size_t smem_acc = static_cast<size_t>(D) * sizeof(double);
+      if (per_head) return WK_ERR_SHAPE;   // rows wider than 8,192 columns take the whole-key fallback only
+      const dim3 grid_a(parts, chunks);
+      const size_t smem_acc = static_cast<size_t>(DF) * sizeof(double);
       if (smem_acc > 200 * 1024) return WK_ERR_SHAPE;
       WK_CUDA_TRY(ctx, cudaFuncSetAttribute(anchor_pass_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             static_cast<int>(smem_acc)));
-      anchor_pass_wide<<<grid_a, kAnchorThreads, smem_acc, s>>>(K, stride, T, D, parts, partial, counters, m64, m32,
+      anchor_pass_wide<<<grid_a, kAnchorThreads, smem_acc, s>>>(K, stride, T, DF, parts, partial, counters, m64, m32,
                                                                 mnorm);
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
-    const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, batch);
-    const size_t smem_m = static_cast<size_t>(D) * sizeof(float);
+    const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, chunks);
+    const size_t smem_m = static_cast<size_t>(DF) * sizeof(float);
     if (per_head)
-      launch_chained(score_pass<true>, grid_s, dim3(kScoreThreads), smem_m, s, K, rm, T, NA, D, m32, s32, scores_out,
+      launch_chained(head_score, grid_s, dim3(kScoreThreads), smem_m, s, K, stride, T, NA, DF, H, m32, s32, scores_out,
                      ctx->status_dev);
     else
-      launch_chained(score_pass<false>, grid_s, dim3(kScoreThreads), smem_m, s, K, rm, T, NA, D, m32, s32, scores_out,
+      launch_chained(score_pass, grid_s, dim3(kScoreThreads), smem_m, s, K, stride, T, NA, DF, m32, s32, scores_out,
                      ctx->status_dev);
     if ((st = after_launch(ctx)) != WK_OK) return st;
   }
