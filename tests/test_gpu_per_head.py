@@ -20,6 +20,8 @@ def _kv(**kw):
     (37, 3, 18, 3, 0.1),          # ragged everything
     (880, 2, 440, 4, 0.1),        # cfg0 shape
     (256, 12, 128, 2, 0.1),       # Matrix-Game head count
+    (880, 12, 440, 3, 0.1),       # the benchmark's chunk shape
+    (1560, 40, 780, 1, 0.05),     # LingBot shape: 40 heads
     (100, 5, 0, 2, 0.1),          # keep nothing
     (100, 5, 200, 2, 0.1),        # keep everything
     (64, 2, 1, 2, 0.05),
