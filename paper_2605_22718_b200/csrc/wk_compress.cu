@@ -27,6 +27,7 @@ constexpr int kMaxAnchorParts = 16;   // slices per problem in the fp64 accumula
 constexpr int kScoreThreads = 256;
 constexpr int kScoreRowsPerCta = 64;
 constexpr int kSelectThreads = 1024;
+constexpr int kSelectThreadsHead = 256;   // per-head problems (128 columns)
 
 __device__ __forceinline__ double bf16_to_f64(uint32_t bits16) {
   return static_cast<double>(__uint_as_float(bits16 << 16));
@@ -435,11 +436,13 @@ __device__ __forceinline__ float key_f32(uint32_t k) {
 }
 
 template <bool kPerHead>
-__global__ void __launch_bounds__(kSelectThreads)
+__global__ void __launch_bounds__(kPerHead ? kSelectThreadsHead : kSelectThreads)
 select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D, int n_keep,
             const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
             int n_norm_parts, int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
   extern __shared__ __align__(16) uint8_t smem[];
+  // a problem of 128 columns has little to do in the refinement: a quarter of the threads, four problems per SM at once
+  constexpr int kThr = kPerHead ? kSelectThreadsHead : kSelectThreads;
   dep_wait();
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem);                       // [NA]
   int32_t* band_idx = reinterpret_cast<int32_t*>(keys + NA);                // [NA]
@@ -447,19 +450,19 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   uint8_t* flag = reinterpret_cast<uint8_t*>(band_s + NA);                  // [NA]
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sel_prefix, sel_rank, n_band, n_below;
-  __shared__ uint32_t warp_tot[kSelectThreads / 32];
-  __shared__ double band_red[8][kSelectThreads / 32];
+  __shared__ uint32_t warp_tot[32];
+  __shared__ double band_red[8][kThr / 32];
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = T + n_keep;
   int32_t* out = keep_idx + static_cast<int64_t>(b) * C;
-  for (int i = tid; i < T; i += kSelectThreads) out[i] = i;                 // the anchor frame is kept whole
+  for (int i = tid; i < T; i += kThr) out[i] = i;                 // the anchor frame is kept whole
   if (n_keep == 0) return;
   if (n_keep == NA) {
-    for (int j = tid; j < NA; j += kSelectThreads) out[T + j] = T + j;
+    for (int j = tid; j < NA; j += kThr) out[T + j] = T + j;
     return;
   }
   const float* sb = s32 + static_cast<int64_t>(b) * NA;
-  for (int j = tid; j < NA; j += kSelectThreads) keys[j] = f32_key(sb[j]);
+  for (int j = tid; j < NA; j += kThr) keys[j] = f32_key(sb[j]);
   if (tid == 0) { sel_prefix = 0; sel_rank = static_cast<uint32_t>(n_keep - 1); n_band = 0; n_below = 0; }
   __syncthreads();
   // radix select: the key of 0-based rank n_keep-1
@@ -468,7 +471,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
     __syncthreads();
     const uint32_t prefix = sel_prefix;
     const uint32_t mask = shift == 24 ? 0u : (0xFFFFFFFFu << (shift + 8));
-    for (int j = tid; j < NA; j += kSelectThreads) {
+    for (int j = tid; j < NA; j += kThr) {
       const uint32_t k = keys[j];
       if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 0xFFu], 1u);
     }
@@ -509,7 +512,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   const double lo = static_cast<double>(theta) - 2.0 * eps;
   const double hi = static_cast<double>(theta) + 2.0 * eps;
   uint32_t my_below = 0;
-  for (int j = tid; j < NA; j += kSelectThreads) {
+  for (int j = tid; j < NA; j += kThr) {
     const double s = static_cast<double>(key_f32(keys[j]));
     uint8_t f = 0;
     if (s < lo) { f = 1; ++my_below; }
@@ -529,7 +532,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   const int vecs = D >> 3;
   for (int t0 = 0; t0 < nb; t0 += 4) {
     double dot[4] = {0.0, 0.0, 0.0, 0.0}, n2[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int v = tid; v < vecs; v += kSelectThreads) {
+    for (int v = tid; v < vecs; v += kThr) {
       double mv[8];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -567,7 +570,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
     __syncthreads();
     if (tid < 4 && t0 + tid < nb) {
       double d = 0.0, n = 0.0;
-      for (int w = 0; w < kSelectThreads / 32; ++w) {
+      for (int w = 0; w < kThr / 32; ++w) {
         d += band_red[2 * tid][w];
         n += band_red[2 * tid + 1][w];
       }
@@ -578,7 +581,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
     __syncthreads();
   }
   // rank the band tokens by (score, index); the `need` lowest are kept
-  for (int t = tid; t < nb; t += kSelectThreads) {
+  for (int t = tid; t < nb; t += kThr) {
     const double s = band_s[t];
     const int idx = band_idx[t];
     int rank = 0;
@@ -590,7 +593,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   }
   __syncthreads();
   // ordered compaction of the kept indices
-  const int per = (NA + kSelectThreads - 1) / kSelectThreads;
+  const int per = (NA + kThr - 1) / kThr;
   const int a0 = min(NA, tid * per), a1 = min(NA, a0 + per);
   uint32_t cnt = 0;
   for (int j = a0; j < a1; ++j) cnt += flag[j];
@@ -603,7 +606,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    uint32_t v = warp_tot[lane];
+    uint32_t v = lane < kThr / 32 ? warp_tot[lane] : 0u;
     uint32_t inc2 = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -688,7 +691,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
                                           static_cast<int>(smem_sel)));
   }
   if (per_head)
-    launch_chained(select_pass<true>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
+    launch_chained(select_pass<true>, dim3(batch), dim3(kSelectThreadsHead), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
                    n_norm_parts, keep_idx, ctx->status_dev);
   else
     launch_chained(select_pass<false>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
