@@ -3,6 +3,7 @@
 ``build_all()`` compiles
   * ``paper_2605_22718_b200/libworldkv.so``  -- the product: the C-ABI library declared in include/wk.h
   * ``wkinputs/libwkinputs.so``              -- the seeded input generators' device side
+  * ``tests/cuda/libwk_wait_probe.so``       -- test-only: the product's bounded mbarrier wait built with a small cap
 with nvcc.  nvcc cross-compiles without a GPU, so this also runs on a CPU-only machine.
 """
 from __future__ import annotations
@@ -16,6 +17,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 CSRC = os.path.join(ROOT, "paper_2605_22718_b200", "csrc")
 LIB_WORLDKV = os.path.join(ROOT, "paper_2605_22718_b200", "libworldkv.so")
 LIB_INPUTS = os.path.join(ROOT, "wkinputs", "libwkinputs.so")
+LIB_WAIT_PROBE = os.path.join(ROOT, "tests", "cuda", "libwk_wait_probe.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
@@ -55,6 +57,9 @@ def build_all(force: bool = False) -> None:
     gen = os.path.join(ROOT, "wkinputs", "gen.cu")
     if force or _stale(LIB_INPUTS, [gen]):
         _run([_nvcc()] + NVCC_FLAGS + ["-o", LIB_INPUTS, gen], "libwkinputs.log")
+    probe = os.path.join(ROOT, "tests", "cuda", "wait_probe.cu")
+    if os.path.exists(probe) and (force or _stale(LIB_WAIT_PROBE, [probe, os.path.join(CSRC, "ptx_sm100.cuh")])):
+        _run([_nvcc()] + NVCC_FLAGS + ["-DWK_WAIT_CAP=4096u", "-o", LIB_WAIT_PROBE, probe], "libwk_wait_probe.log")
 
 
 if __name__ == "__main__":

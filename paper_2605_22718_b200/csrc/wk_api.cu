@@ -140,6 +140,19 @@ static wk_status check_config(const wk_config* c) {
   return WK_OK;
 }
 
+// Every entry point that touches the device runs on the context's own device, whatever the caller had current.
+static wk_status use_device(wk_ctx* ctx) {
+  int dev = -1;
+  WK_CUDA_TRY(ctx, cudaGetDevice(&dev));
+  if (dev != ctx->cfg.device) WK_CUDA_TRY(ctx, cudaSetDevice(ctx->cfg.device));
+  return WK_OK;
+}
+#define WK_USE_DEVICE(ctx)                                  \
+  do {                                                      \
+    wk_status st__ = ::wk::use_device(ctx);                 \
+    if (st__ != WK_OK) return st__;                         \
+  } while (0)
+
 }  // namespace wk
 
 using namespace wk;
@@ -190,6 +203,7 @@ wk_status wk_bind(wk_ctx* ctx, void* pool_dev, size_t pool_bytes, void* scratch_
   if (!ctx || !pool_dev || !scratch_dev) return WK_ERR_ARG;
   if ((reinterpret_cast<uintptr_t>(pool_dev) & 255u) || (reinterpret_cast<uintptr_t>(scratch_dev) & 255u)) return WK_ERR_ARG;
   if (max_batch < 0 || max_lq < 0 || max_splits < 0) return WK_ERR_ARG;
+  WK_USE_DEVICE(ctx);
   PoolLayout pl = pool_layout(ctx->cfg);
   ScratchLayout sl = scratch_layout(ctx->cfg, max_batch, max_lq, max_splits);
   if (pool_bytes < pl.total || scratch_bytes < sl.total) return WK_ERR_SHAPE;
@@ -226,6 +240,7 @@ wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_str
                             int32_t* keep_idx_out, float* scores_out, void* stream) {
   if (!ctx || !K_chunks || !keep_idx_out || batch < 0) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (!aligned16(K_chunks) || (batch_stride_elems & 7) != 0) return WK_ERR_ARG;
   if (batch > 1 && batch_stride_elems < static_cast<int64_t>(ctx->FT) * ctx->D) return WK_ERR_ARG;
   if (batch > ctx->max_batch) return WK_ERR_SHAPE;
@@ -239,6 +254,7 @@ wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_c
                          int64_t chunk_tag, int32_t* slot_io_host, void* stream) {
   if (!ctx || !K_chunks || !V_chunks || !keep_idx_dev || !pose_host || !slot_io_host) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (!aligned16(K_chunks) || !aligned16(V_chunks) || (batch_stride_elems & 7) != 0) return WK_ERR_ARG;
   if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers) return WK_ERR_SHAPE;
   if (n > 1 && batch_stride_elems < static_cast<int64_t>(ctx->FT) * ctx->D) return WK_ERR_ARG;
@@ -287,6 +303,7 @@ size_t wk_host_chunk_bytes(const wk_ctx* ctx) {
 wk_status wk_pool_store_host(wk_ctx* ctx, int32_t slot, void* host_dst, void* stream) {
   if (!ctx || !host_dst) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (slot < 0 || slot >= ctx->cfg.pool_slots || ctx->slots[slot].state != SLOT_VALID) return WK_ERR_BAD_SLOT;
   // one layer of one slot is contiguous (C * D elements); the layers of a slot are pool_slots such blocks apart
   const size_t row = static_cast<size_t>(ctx->C) * ctx->D * sizeof(__nv_bfloat16);
@@ -305,6 +322,7 @@ wk_status wk_pool_load_host(wk_ctx* ctx, int32_t layer0, int32_t n, const void* 
                             int64_t chunk_tag, int32_t* slot_io_host, void* stream) {
   if (!ctx || !host_src || !pose_host || !slot_io_host) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers) return WK_ERR_SHAPE;
   int slot = *slot_io_host;
   if (slot < 0) {
@@ -351,6 +369,7 @@ wk_status wk_pool_load_host(wk_ctx* ctx, int32_t layer0, int32_t n, const void* 
 wk_status wk_pool_evict(wk_ctx* ctx, int32_t slot, void* stream) {
   if (!ctx) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (slot < 0 || slot >= ctx->cfg.pool_slots || ctx->slots[slot].state != SLOT_VALID) return WK_ERR_BAD_SLOT;
   wk_status st = launch_slot_mark(ctx, slot, 0, ctx->slots[slot].pose, static_cast<cudaStream_t>(stream));
   if (st != WK_OK) return st;
@@ -384,6 +403,7 @@ wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_
                       int32_t* n_out_host, void* stream) {
   if (!ctx || !cur_pose_host || !slots_out_dev || !n_out_host) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (k < 0 || k > ctx->cfg.max_k) return WK_ERR_SHAPE;
   const int M = wk_pool_count(ctx);
   *n_out_host = k < M ? k : M;
@@ -399,6 +419,7 @@ wk_status wk_retrieve_scan(wk_ctx* ctx, const float* poses_dev, const int32_t* v
   if (!aligned16(poses_dev) || !aligned16(scratch_dev)) return WK_ERR_ARG;
   if (k < 0 || k > 64 || k > out_capacity || n < 0 || n >= (int64_t(1) << 31)) return WK_ERR_SHAPE;
   if (scratch_bytes < retrieve_scan_scratch_bytes()) return WK_ERR_SHAPE;
+  WK_USE_DEVICE(ctx);
   return launch_retrieve_scan(ctx, poses_dev, valid_dev, n, cur_pose_host, k, ids_out_dev, dist_out_dev, out_capacity,
                               scratch_dev, static_cast<cudaStream_t>(stream));
 }
@@ -407,6 +428,7 @@ wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t l
                             float* score_out_dev, int32_t* n_out_host, void* stream) {
   if (!ctx || !Q || !slots_out_dev || !n_out_host || lq < 1) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (!aligned16(Q)) return WK_ERR_ARG;
   if (layer < 0 || layer >= ctx->cfg.n_layers || lq > ctx->max_lq || k < 0 || k > ctx->cfg.max_k) return WK_ERR_SHAPE;
   if (ctx->cfg.pool_slots > 1024) return WK_ERR_SHAPE;
@@ -421,6 +443,7 @@ wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t
                               int32_t kv_splits, void* stream) {
   if (!ctx || !Q || !O || lq < 1 || n_segs < 0 || n_slots < 0) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   if (n_segs == 0 && n_slots == 0) return WK_ERR_ARG;
   if ((n_segs > 0 && !segs_host) || (n_slots > 0 && !slots_dev)) return WK_ERR_ARG;
   if (!aligned16(Q) || !aligned16(O)) return WK_ERR_ARG;
@@ -438,6 +461,7 @@ wk_status wk_memory_attention(wk_ctx* ctx, int32_t layer, const void* Q, int32_t
 wk_status wk_poll_status(wk_ctx* ctx, uint32_t* device_flags, void* stream) {
   if (!ctx) return WK_ERR_ARG;
   if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   uint32_t flags = 0;
   WK_CUDA_TRY(ctx, cudaMemcpyAsync(&flags, ctx->status_dev, sizeof(flags), cudaMemcpyDeviceToHost, s));

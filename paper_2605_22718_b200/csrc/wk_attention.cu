@@ -313,10 +313,12 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
       walk.init(p);
       Piece pc;
       uint32_t jk = 0, n = 0;
+      uint32_t armed_q = 0, armed_k = 0, armed_v = 0;   // loads armed so far (a barrier's u-th use completes its phase u)
       bool ok = true;
       while (ok && walk.next(p, pc)) {
         if (!(ok = wait_or_abort(&bars.q_empty, (n & 1) ^ 1, &s_abort, p.status))) break;
         mbar_expect_tx(&bars.q_full, 2 * kTileBytes);
+        armed_q = n + 1;
         for (int i = 0; i < 2; ++i)
           for (int half = 0; half < 2; ++half)
             tma_load_2d(sQ + i * kTileBytes + half * kHalfTileBytes, &p.tm_q, &bars.q_full, pc.h * kHeadDim + half * 64,
@@ -331,6 +333,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           const uint32_t phk = (jk / kStagesK) & 1, ph = (jk / kStagesV) & 1;
           if (!(ok = wait_or_abort(&bars.k_empty[sk], phk ^ 1, &s_abort, p.status))) break;
           mbar_expect_tx(&bars.k_full[sk], kTileBytes);
+          armed_k = jk + 1;
           uint8_t* dk = sK + sk * kTileBytes;
           if (ti.seg >= 0) {
             tma_load_2d(dk, &p.tm_kd[ti.seg], &bars.k_full[sk], x, ti.row0);
@@ -342,6 +345,7 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           if (kLse) { ++jk; continue; }   // no P V product: V is not fetched
           if (!(ok = wait_or_abort(&bars.v_empty[st], ph ^ 1, &s_abort, p.status))) break;
           mbar_expect_tx(&bars.v_full[st], kTileBytes);
+          armed_v = jk + 1;
           uint8_t* dv = sV + st * kTileBytes;
           if (ti.seg >= 0) {
             tma_load_2d(dv, &p.tm_vd[ti.seg], &bars.v_full[st], x, ti.row0);
@@ -354,14 +358,19 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
         }
         ++n;
       }
-      // Do not leave while copies may still be landing in shared memory: wait (bounded) for the loads issued last.
+      // After an abort the consumers no longer wait for the tiles in flight, so this thread does: a CTA must not free
+      // its shared memory under copies that are still landing.  Per stage, the load armed last is use u = (count - 1 -
+      // stage) / stages of that stage's barrier, whose phase u has parity u & 1; a stage that was never armed is skipped.
       if (s_abort) {
-        for (int s = 0; s < kStagesK; ++s)
+        auto drain = [](uint64_t* bar, uint32_t use) {
           for (uint32_t i = 0; i < (1u << 16); ++i)
-            if (mbar_try_wait(&bars.k_full[s], 0) || mbar_try_wait(&bars.k_full[s], 1)) break;
-        for (int s = 0; s < kStagesV; ++s)
-          for (uint32_t i = 0; i < (1u << 16); ++i)
-            if (mbar_try_wait(&bars.v_full[s], 0) || mbar_try_wait(&bars.v_full[s], 1)) break;
+            if (mbar_try_wait(bar, use & 1)) break;
+        };
+        if (armed_q > 0) drain(&bars.q_full, armed_q - 1);
+        for (uint32_t s = 0; s < kStagesK; ++s)
+          if (armed_k > s) drain(&bars.k_full[s], (armed_k - 1 - s) / kStagesK);
+        for (uint32_t s = 0; s < kStagesV; ++s)
+          if (armed_v > s) drain(&bars.v_full[s], (armed_v - 1 - s) / kStagesV);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -727,13 +736,12 @@ int attention_partial_slots(int n_heads, int max_lq, int max_splits) {
 wk_status launch_attention(wk_ctx* ctx, int layer, const __nv_bfloat16* Q, int lq, const wk_dense_seg* segs, int n_segs,
                            const int32_t* slots_dev, int n_slots, __nv_bfloat16* O, float* lse, int kv_splits,
                            cudaStream_t s, bool lse_only) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  if (!ctx->attn_attr_set) {   // the attribute belongs to the device the context lives on
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(kSmemBytes)));
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(memory_attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(kSmemBytes)));
-    attr_set = true;
+    ctx->attn_attr_set = true;
   }
   AttnParams p;
   wk_status st = encode_rows_map(ctx, Q, lq, kTileQ, &p.tm_q);

@@ -361,7 +361,7 @@ score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
     if (lane < 2 && (lane == 0 || has_b)) {
       const float dot = lane ? dot_b : dot_a, n2 = lane ? n2_b : n2_a;
       const int jj = lane ? jb : j;
-      const float sc = n2 > 0.f ? __fdiv_rn(dot, __fsqrt_rn(n2)) : 0.f;
+      const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
       if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
       s32[static_cast<int64_t>(b) * NA + jj] = sc;
       if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
@@ -413,7 +413,7 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
         n2 = half_warp_sum(n2);
         const int head = v >> 4;
         if ((lane & 15) == 0 && head < H) {
-          const float sc = n2 > 0.f ? __fdiv_rn(dot, __fsqrt_rn(n2)) : 0.f;
+          const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
           if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
           const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + j;
           s32[at] = sc;
@@ -574,7 +574,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
         d += band_red[2 * tid][w];
         n += band_red[2 * tid + 1][w];
       }
-      const double sc = n > 0.0 ? d / sqrt(n) : 0.0;
+      const double sc = n == 0.0 ? 0.0 : d / sqrt(n);
       if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
       band_s[t0 + tid] = sc;
     }

@@ -76,6 +76,8 @@ struct wk_ctx {
   CUtensorMap tm_kpool, tm_vpool;
   std::vector<wk::TmapKey> tmap_cache;
   size_t tmap_cache_next = 0;
+  // per-context (hence per-device) one-time kernel attributes: opt-ins to large dynamic shared memory
+  bool attn_attr_set = false;
   // diagnostics
   int32_t last_cuda_error = 0;
   int64_t launches = 0;

@@ -26,7 +26,7 @@ __device__ __forceinline__ double block_max(double v, double* red) {
 __global__ void __launch_bounds__(kRetrieveThreads)
 retrieve_kernel(const float* __restrict__ poses, const int32_t* __restrict__ valid, int n_slots, Pose8 cur, int k,
                 int max_k, double* __restrict__ dist /*[2][n_slots]*/, int32_t* __restrict__ slots_out,
-                double* __restrict__ dist_out) {
+                double* __restrict__ dist_out, uint32_t* __restrict__ status /*may be null*/) {
   __shared__ double red[kRetrieveThreads / 32];
   const int tid = threadIdx.x;
   double* dt = dist;
@@ -41,6 +41,11 @@ retrieve_kernel(const float* __restrict__ poses, const int32_t* __restrict__ val
     const double t = dx * dx + dy * dy + dz * dz;
     const double dot = static_cast<double>(p[4]) * cur.v[4] + static_cast<double>(p[5]) * cur.v[5] +
                        static_cast<double>(p[6]) * cur.v[6] + static_cast<double>(p[7]) * cur.v[7];
+    if (!isfinite(t) || !isfinite(dot)) {          // a NaN/Inf pose (stored or current) is not a candidate
+      dt[s] = -1.0;
+      if (status) atomicOr(status, WK_DEV_NONFINITE);
+      continue;
+    }
     const double r = 2.0 * acos(fmin(1.0, fabs(dot)));    // q and -q are the same rotation
     dt[s] = t;
     dr[s] = r;
@@ -159,7 +164,7 @@ wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* sl
   for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose[i];
   double* dist = reinterpret_cast<double*>(ctx->scratch_base + ctx->sl.dist_off);
   retrieve_kernel<<<1, kRetrieveThreads, 0, s>>>(ctx->poses_dev, ctx->valid_dev, ctx->cfg.pool_slots, cur, k,
-                                                 ctx->cfg.max_k, dist, slots_out, dist_out);
+                                                 ctx->cfg.max_k, dist, slots_out, dist_out, ctx->status_dev);
   return after_launch(ctx);
 }
 
@@ -203,6 +208,6 @@ extern "C" wk_status wk_retrieve_noalloc(const float* poses_dev, const int32_t* 
   Pose8 cur;
   for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose_host[i];
   retrieve_kernel<<<1, kRetrieveThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-      poses_dev, valid_dev, n_slots, cur, k, max_k, scratch_of_device[dev], slots_out_dev, dist_out_dev);
+      poses_dev, valid_dev, n_slots, cur, k, max_k, scratch_of_device[dev], slots_out_dev, dist_out_dev, nullptr);
   return cudaGetLastError() == cudaSuccess ? WK_OK : WK_ERR_CUDA;
 }
