@@ -233,8 +233,8 @@ class ChunkStepBench:
                 segs = [(curK[l], curV[l])]
                 if w.window_frames > 0:
                     rows = self.winK.shape[1] // w.window_segments
-                    for i in range(w.window_segments):
-                        segs.append((self.winK[l, i * rows:(i + 1) * rows], self.winV[l, i * rows:(i + 1) * rows]))
+                    for q in range(w.window_segments):
+                        segs.append((self.winK[l, q * rows:(q + 1) * rows], self.winV[l, q * rows:(q + 1) * rows]))
                 kv.memory_attention(l, Q[l, s], segs, self.slots, n, O=O[l, s], kv_splits=self.kv_splits)
         if record_attention_events:
             e1.record()

@@ -316,7 +316,10 @@ def memory_attention(Q, dense_segments, pool: Optional[PoolModel], layer: int, s
 
 
 def query_scores(Q, pool: PoolModel, layer: int, scale: Optional[float] = None):
-    """Returns (slots ascending, score per slot).  Scores are non-negative and sum to 1."""
+    """Returns (slots ascending, score per slot).  Scores are non-negative and sum to 1.
+
+    Reading R12 written out: per head and query row ONE softmax over all stored keys of the layer; a chunk's mass is
+    the sum of the weights of its own keys; its score is the mean of that mass over heads and rows."""
     slots = pool.valid_slots()
     Qf = _as_f64(Q)
     Lq, H, d = Qf.shape
@@ -324,17 +327,16 @@ def query_scores(Q, pool: PoolModel, layer: int, scale: Optional[float] = None):
         scale = 1.0 / np.sqrt(d)
     if not slots:
         return slots, np.zeros(0)
-    lse = np.empty((len(slots), H, Lq))
-    for n, s in enumerate(slots):
-        Ks = _as_f64(pool.K[(layer, s)])
-        for h in range(H):
-            S = scale * (Qf[:, h, :] @ Ks[:, h, :].T)               # [Lq, C]
-            mx = S.max(axis=1)
-            lse[n, h] = mx + np.log(np.exp(S - mx[:, None]).sum(axis=1))
-    top = lse.max(axis=0)
-    w = np.exp(lse - top)                                            # [M, H, Lq]
-    mass = w / w.sum(axis=0)                                         # softmax mass of each chunk, per head and row
-    return slots, mass.mean(axis=(1, 2))
+    Kall = np.concatenate([_as_f64(pool.K[(layer, s)]) for s in slots], axis=0)       # [sum of C, H, d]
+    owner = np.concatenate([np.full(pool.K[(layer, s)].shape[0], n) for n, s in enumerate(slots)])
+    score = np.zeros(len(slots))
+    for h in range(H):
+        S = scale * (Qf[:, h, :] @ Kall[:, h, :].T)                  # [Lq, all stored keys]
+        W = np.exp(S - S.max(axis=1, keepdims=True))
+        W /= W.sum(axis=1, keepdims=True)                            # softmax over every stored key
+        for n in range(len(slots)):
+            score[n] += W[:, owner == n].sum()                       # the chunk's share, summed over the rows
+    return slots, score / (H * Lq)
 
 
 def retrieve_query(Q, pool: PoolModel, layer: int, k: int, scale: Optional[float] = None):

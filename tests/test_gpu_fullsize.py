@@ -90,6 +90,21 @@ def check_sampled_attention(w, layer, O, lse, q_stream, dense_specs, slot_chunks
     return worst_abs, worst_rel
 
 
+def oracle_keep_set(w, layer, chunk, cache=None):
+    """The oracle's keep-set of one generated chunk.  Its full-width keys are drawn by the device side of the seeded
+    input generator (bit-identical to the numpy side, see test_device_generators_match_numpy), which at D = 5,120 is far
+    quicker than numpy; the scores, the selection and the margin are the oracle's."""
+    if cache is not None and chunk in cache:
+        return cache[chunk]
+    tmp = torch.empty((w.F * w.T, w.D), dtype=torch.bfloat16, device="cuda")
+    wd.key_chunk(tmp, w.seed, layer, chunk, w.T, w.D, w.sigma, w.F)
+    idx, _, m = o.compress_chunk(wd.to_host_bits(tmp), w.T, w.n_keep)
+    assert m > 1e-11
+    if cache is not None:
+        cache[chunk] = idx
+    return idx
+
+
 SAMPLE_ROWS = {2640: [0, 1, 127, 128, 255, 256, 1333, 2559, 2560, 2639],
                4680: [0, 127, 128, 2300, 4607, 4608, 4679]}
 
@@ -127,11 +142,12 @@ def test_cfg1_matrix_game_single_layer():
     assert float((O2.float() - O.float()).abs().max()) <= 2e-3
 
 
-def test_paper_default_window_matrix_game_shape():
+@pytest.mark.parametrize("name,heads", [("paper_mg", [2, 9]), ("paper_lb", [0, 23, 39])])
+def test_paper_default_window_both_model_shapes(name, heads):
     """Section 5.1's window: sink 3 + retrieved 9 (six compressed chunks) + recent 3 + denoising 3 = 18 latent frames,
-    passed as three dense segments plus six pool slots."""
+    passed as three dense segments plus six pool slots, at 880 (12 heads) and 1,560 (40 heads) tokens per frame."""
     from paper_2605_22718_b200 import WorldKV
-    w = wi.WORKLOADS["paper_mg"]
+    w = wi.WORKLOADS[name]
     assert w.Lkv == 18 * w.T
     kv = WorldKV(n_layers=1, n_heads=w.n_heads, tokens_per_frame=w.T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
                  max_k=w.k, max_batch=1, max_lq=w.Lq, max_splits=2, max_dense_segments=3)
@@ -144,10 +160,8 @@ def test_paper_default_window_matrix_game_shape():
     np.testing.assert_array_equal(slots.cpu().numpy()[:n], ref_slots)
     keep_of = {}
     for c in ref_slots.tolist():
-        idx, _, m = o.compress_chunk(wi.key_chunk_bf16(w.seed, 0, c, w.T, w.D, w.sigma), w.T, w.n_keep)
-        assert m > 1e-11
-        np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), idx)
-        keep_of[c] = idx
+        keep_of[c] = oracle_keep_set(w, 0, c)
+        np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), keep_of[c])
     Q = torch.empty((w.Lq, w.n_heads, 128), dtype=torch.bfloat16, device="cuda")
     wd.query(Q, w.seed, 0, 0, cur_chunk)
     cur = dense_rows_device(w, 0, [cur_chunk], w.Lq)
@@ -158,7 +172,7 @@ def test_paper_default_window_matrix_game_shape():
     assert kv.poll_status() == (0, 0)
     check_sampled_attention(w, 0, O, lse, (0, cur_chunk),
                             [([w.pool_chunks + 4], 3 * w.T), ([w.pool_chunks + 1], 3 * w.T), ([cur_chunk], w.Lq)],
-                            ref_slots.tolist(), keep_of, heads=[2, 9], rows=SAMPLE_ROWS[w.Lq])
+                            ref_slots.tolist(), keep_of, heads=heads, rows=SAMPLE_ROWS[w.Lq])
 
 
 def test_cfg3_lingbot_single_layer_and_k_sweep():
@@ -173,7 +187,7 @@ def test_cfg3_lingbot_single_layer_and_k_sweep():
     wd.query(Q, w.seed, 0, 0, cur_chunk)
     cur = dense_rows_device(w, 0, [cur_chunk], w.Lq)
     win = dense_rows_device(w, 0, [w.pool_chunks, w.pool_chunks + 1], w.window_frames * w.T)
-    lses = {}
+    lses, keep_cache = {}, {}
     for k in w.k_sweep:
         slots, n = kv.retrieve(poses[cur_chunk], k)
         ref_slots, _, margin = o.retrieve(poses[cur_chunk], poses[:w.pool_chunks], list(range(w.pool_chunks)), k)
@@ -184,16 +198,15 @@ def test_cfg3_lingbot_single_layer_and_k_sweep():
         assert kv.poll_status() == (0, 0)
         assert torch.isfinite(O.float()).all()
         lses[k] = lse.clone()
-        if k == 2:      # the oracle leg: two retrieved chunks, full width for the keep-set
-            keep_of = {}
-            for c in ref_slots.tolist():
-                idx, _, m = o.compress_chunk(wi.key_chunk_bf16(w.seed, 0, c, w.T, w.D, w.sigma), w.T, w.n_keep)
-                assert m > 1e-11
-                np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), idx)
-                keep_of[c] = idx
-            check_sampled_attention(w, 0, O, lse, (0, cur_chunk),
-                                    [([cur_chunk], w.Lq), ([w.pool_chunks, w.pool_chunks + 1], w.window_frames * w.T)],
-                                    ref_slots.tolist(), keep_of, heads=[0, 39], rows=SAMPLE_ROWS[w.Lq])
+        # the oracle leg at every budget: the retrieved chunks' keep-sets (full width) bit-exact, then sampled rows --
+        # two heads and seven rows at k = 2, one head and four rows at the larger budgets
+        for c in ref_slots.tolist():
+            idx = oracle_keep_set(w, 0, c, keep_cache)
+            np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), idx)
+        heads, rows = ([0, 39], SAMPLE_ROWS[w.Lq]) if k == 2 else ([(7 * k) % w.n_heads], [0, 128, 2300, 4679])
+        check_sampled_attention(w, 0, O, lse, (0, cur_chunk),
+                                [([cur_chunk], w.Lq), ([w.pool_chunks, w.pool_chunks + 1], w.window_frames * w.T)],
+                                ref_slots.tolist(), keep_cache, heads=heads, rows=rows)
         if k == 8:      # properties that hold at any size: slot order does not matter
             rev = torch.flip(slots[:n], dims=[0]).contiguous()
             O_rev = kv.memory_attention(0, Q, [win, cur], rev, n)
@@ -232,6 +245,37 @@ def test_cfg4_full_uncompressed_history_and_kv_splits():
     for splits in (1, 4, 16):
         assert float((outs[splits][0].float() - O.float()).abs().max()) <= 2e-3
         assert float((outs[splits][1] - lse).abs().max()) <= 2e-3
+
+
+def test_cfg4c_compressed_history_and_kv_splits():
+    """The one-minute history with every chunk compressed to 50 %: 125 x 1,320 = 165,000 stored tokens, all attended
+    (plus the 2,640 of the denoising chunk).  All 125 keep-sets are compared with the oracle's; sampled rows at every
+    KV split against the oracle."""
+    from paper_2605_22718_b200 import WorldKV
+    w = wi.WORKLOADS["cfg4c"]
+    kv = WorldKV(n_layers=1, n_heads=w.n_heads, tokens_per_frame=w.T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
+                 max_k=w.pool_chunks, max_batch=1, max_lq=w.Lq, max_splits=16)
+    assert w.pool_chunks * w.C == 165000 and 2 * w.C == 3 * w.T
+    poses = wi.loop_poses(w.seed, w.pool_chunks + 3)
+    keeps = fill_pool_on_device(kv, w, poses)
+    keep_of = {}
+    for c in range(w.pool_chunks):
+        keep_of[c] = oracle_keep_set(w, 0, c)
+        np.testing.assert_array_equal(keeps[c, 0].cpu().numpy(), keep_of[c])
+    cur_chunk = w.pool_chunks + 2
+    slots, n = kv.retrieve(poses[cur_chunk], w.pool_chunks)
+    ref_slots, _, _ = o.retrieve(poses[cur_chunk], poses[:w.pool_chunks], list(range(w.pool_chunks)), w.pool_chunks)
+    assert n == w.pool_chunks
+    np.testing.assert_array_equal(slots.cpu().numpy(), ref_slots)
+    Q = torch.empty((w.Lq, w.n_heads, 128), dtype=torch.bfloat16, device="cuda")
+    wd.query(Q, w.seed, 0, 0, cur_chunk)
+    cur = dense_rows_device(w, 0, [cur_chunk], w.Lq)
+    for splits, head in ((0, 5), (1, 0), (4, 11), (16, 7)):
+        lse = torch.empty((w.n_heads, w.Lq), dtype=torch.float32, device="cuda")
+        O = kv.memory_attention(0, Q, [cur], slots, n, lse_out=lse, kv_splits=splits)
+        assert kv.poll_status() == (0, 0)
+        check_sampled_attention(w, 0, O, lse, (0, cur_chunk), [([cur_chunk], w.Lq)], ref_slots.tolist(), keep_of,
+                                heads=[head], rows=[0, 129, 1300, 2639])
 
 
 def test_cfg2_chunk_step_in_the_bench_configuration():

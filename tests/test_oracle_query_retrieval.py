@@ -13,25 +13,41 @@ def _pool(keys_per_chunk, H=2, d=8):
     return pool
 
 
-def test_mass_is_the_sum_of_softmax_weights_over_the_chunk():
-    """Independent route: one softmax over the concatenation of all stored keys, weights added per chunk."""
+def test_mass_through_per_chunk_log_sum_exp():
+    """Independent route to the same numbers: a log-sum-exp per stored chunk, then a softmax over the chunks' values
+    (exp(lse_c) is the chunk's un-normalised mass, so normalising over chunks gives its share)."""
     rng = np.random.default_rng(0)
     H, d, Lq = 2, 8, 5
     chunks = [rng.standard_normal((n, H, d)) * 2 for n in (3, 7, 4, 6)]
     pool = _pool(chunks, H, d)
     Q = rng.standard_normal((Lq, H, d))
     slots, score = o.query_scores(Q, pool, 0)
-    Kall = np.concatenate(chunks)
-    owner = np.concatenate([np.full(len(c), i) for i, c in enumerate(chunks)])
-    expect = np.zeros(4)
-    for h in range(H):
-        S = (Q[:, h] @ Kall[:, h].T) / np.sqrt(d)
-        W = np.exp(S - S.max(1, keepdims=True))
-        W /= W.sum(1, keepdims=True)
-        for i in range(4):
-            expect[i] += W[:, owner == i].sum()
-    np.testing.assert_allclose(score, expect / (H * Lq), atol=1e-14)
+    lse = np.empty((4, H, Lq))
+    for c, K in enumerate(chunks):
+        for h in range(H):
+            S = (Q[:, h] @ K[:, h].T) / np.sqrt(d)
+            mx = S.max(axis=1)
+            lse[c, h] = mx + np.log(np.exp(S - mx[:, None]).sum(axis=1))
+    w = np.exp(lse - lse.max(axis=0))
+    expect = (w / w.sum(axis=0)).mean(axis=(1, 2))
+    np.testing.assert_allclose(score, expect, atol=1e-14)
     assert abs(score.sum() - 1) < 1e-14 and slots == [0, 1, 2, 3]
+
+
+def test_mass_brute_force_loops():
+    """The definition with explicit loops on a tiny case: every (head, row) normalises over all stored keys."""
+    rng = np.random.default_rng(5)
+    H, d, Lq = 1, 4, 2
+    chunks = [rng.standard_normal((n, H, d)) for n in (2, 3)]
+    pool = _pool(chunks, H, d)
+    Q = rng.standard_normal((Lq, H, d))
+    expect = np.zeros(2)
+    for r in range(Lq):
+        logits = [[float(Q[r, 0] @ k[0]) / np.sqrt(d) for k in K] for K in chunks]
+        Z = sum(np.exp(x) for row in logits for x in row)
+        for c in range(2):
+            expect[c] += sum(np.exp(x) for x in logits[c]) / Z
+    np.testing.assert_allclose(o.query_scores(Q, pool, 0)[1], expect / Lq, atol=1e-14)
 
 
 def test_closed_forms():

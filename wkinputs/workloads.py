@@ -89,4 +89,7 @@ WORKLOADS = {
     # full-KV stress: the whole uncompressed one-minute history (125 x 2,640 = 330,000 tokens)
     "cfg4": Workload("cfg4", seed=4, n_layers=1, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
                      window_frames=0, n_keep=1760, pool_chunks=125, k=125, sigma=0.1, trajectory="loop"),
+    # the same one-minute history with every chunk compressed to 50 % (125 x 1,320 = 165,000 tokens), all of it attended
+    "cfg4c": Workload("cfg4c", seed=4, n_layers=1, n_heads=12, head_dim=128, T=880, F=3, q_frames=3,
+                      window_frames=0, n_keep=440, pool_chunks=125, k=125, sigma=0.1, trajectory="loop"),
 }
