@@ -30,7 +30,7 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   // size, the per-problem ones grow by n_heads
   const size_t Bc = static_cast<size_t>(max_batch > 0 ? max_batch : 1);
   const size_t B = Bc * (c.score_mode == WK_SCORE_PER_HEAD ? c.n_heads : 1);
-  s.anchor_parts = 16;
+  s.anchor_parts = 32;
   size_t off = 0;
   s.m32_off = off;   off += align_up(Bc * D * sizeof(float), 256);
   s.m64_off = off;   off += align_up(Bc * D * sizeof(double), 256);
@@ -38,7 +38,7 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   s.mnorm_off = off; off += align_up(B * 32 * sizeof(double), 256);   // up to 32 shares of |m|^2 per problem
   s.part_off = off;  off += align_up(Bc * s.anchor_parts * D * sizeof(double), 256);
   s.inv_off = off;   off += align_up(B * c.tokens_per_frame * sizeof(double), 256);
-  s.cnt_off = off;   off += align_up(B * sizeof(uint32_t), 256);
+  s.cnt_off = off;   off += align_up(2 * Bc * sizeof(uint32_t), 256);   // tickets of the anchor and the score pass
   s.dist_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * 2 * sizeof(double), 256);
   const size_t slots = static_cast<size_t>(attention_partial_slots(c.n_heads, max_lq > 0 ? max_lq : 1, max_splits));
   s.opart_off = off;   off += align_up(slots * 2 * kTileQ * kHeadDim * sizeof(float), 256);

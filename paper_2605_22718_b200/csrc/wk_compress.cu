@@ -4,30 +4,30 @@
 // The mean over anchors is pulled inside the dot product: s_j = (k_j . m) / |k_j| with
 // m = (1/T) sum_i a_i / |a_i|, so a chunk is read exactly once (3T*D bf16) instead of T^2 times.
 //
-//   anchor_norms, anchor_accumulate
-//                 read the T anchor rows (the second time from L2): fp64 row norms, then m in fp64 with thread-owned
-//                 columns; the per-CTA slices are added in a fixed order -> m64, m32 = fp32(m64), |m|
-//   score_pass    reads the (F-1)T non-anchor rows once, fp32 dot with the shared-memory-staged m32 and fp32
-//                 norm, warp-shuffle reductions -> s32
-//   select_pass   per problem: the n_keep-th smallest s32 (radix select) is the threshold; tokens further than
-//                 a proved fp32 error band from it are decided at once, the few inside the band are re-scored
-//                 in fp64 against m64 and ranked exactly by (score, index); emits the ascending index list
+//   anchor_pass   reads the T anchor rows once: groups of rows arrive in shared memory by bulk copy (double-buffered),
+//                 a warp takes the fp64 norm of a row, then every thread adds a_i / |a_i| for the columns it owns, in
+//                 fp64, over the rows of the group.  A CTA covers one slice of one problem's rows; the last CTA of a
+//                 problem (atomic ticket, nobody waits) adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|^2
+//   score_select  reads the (F-1)T non-anchor rows once: fp32 dot with the shared-memory-staged m32 and fp32 norm,
+//                 warp-shuffle reductions -> s32.  The CTA that finishes a problem's last rows (ticket again) runs that
+//                 problem's selection while the other CTAs are still streaming later problems:
+//   selection     the n_keep-th smallest s32 (radix select) is the threshold; tokens further than a proved fp32 error
+//                 band from it are decided at once, the few inside the band are re-scored in fp64 against m64 and
+//                 ranked exactly by (score, index); emits the ascending index list
+// Per-head keys (one keep-set per head) use the same anchor_pass with per-head norms, then head_score and a
+// selection launch of its own (n_heads problems per chunk).
 //
 // The selection is therefore decided in fp64 wherever fp32 could not decide it, and is reproducible
 // run to run (no floating-point atomics anywhere).
+#include "ptx_sm100.cuh"
 #include "wk_internal.cuh"
 
 namespace wk {
 namespace {
 
-constexpr int kAnchorThreads = 256;
-constexpr int kColSplit = 2;          // column halves per row slice in the fp64 accumulation
-constexpr int kMaxNormParts = 32;     // |m|^2 arrives in up to this many per-CTA shares per problem (D <= 16384)
-constexpr int kMaxAnchorParts = 16;   // slices per problem in the fp64 accumulation (matches the scratch layout)
+constexpr int kMaxNormParts = 32;     // pitch of the per-problem |m|^2 record in scratch (one share is used)
 constexpr int kScoreThreads = 256;
-constexpr int kScoreRowsPerCta = 64;
-constexpr int kSelectThreads = 1024;
-constexpr int kSelectThreadsHead = 256;   // per-head problems (128 columns)
+constexpr int kScoreRowsPerCta = 32;
 
 __device__ __forceinline__ double bf16_to_f64(uint32_t bits16) {
   return static_cast<double>(__uint_as_float(bits16 << 16));
@@ -46,13 +46,12 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// The five kernels of one call depend on each other in a chain and are launched with launch_chained (wk_internal.cuh):
+// The kernels of one call depend on each other in a chain and are launched with launch_chained (wk_internal.cuh):
 // nothing is read or written before dep_wait(), so only launch latency and block scheduling overlap.
 
 // Where the rows of problem b live.  A chunk is [F*T][rs] bf16; with whole-token keys (one keep-set per chunk) a
 // problem is a chunk and D = rs; with per-head keys a chunk holds hs = n_heads problems, problem (chunk, h) owning
 // columns [h*D, (h+1)*D) of every row, D = head_dim.
-// The kernels are instantiated for both cases, so that the whole-key case keeps its plain arithmetic (row pitch = D).
 struct RowMap {
   int64_t stride;   // elements between chunks
   int rs;           // elements between token rows
@@ -66,44 +65,6 @@ struct RowMap {
   __device__ __forceinline__ int pitch(int D) const { return kPerHead ? rs : D; }
 };
 
-// ------------------------------------------------------------------------------------------------
-// anchor pass, two streaming kernels with no block barrier in their loops.
-//   anchor_norms:      one warp per anchor row, fp64 squared norm -> 1/|a_i| (0 for a zero key)
-//   anchor_accumulate: grid = (parts * kColSplit, batch), block = D/(8 kColSplit) threads; a thread owns 8 columns and adds
-//                      a_i[8t..] / |a_i| over the rows of its slice in fp64; the anchor rows come from L2 the second
-//                      time.  The last CTA of a problem adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|.
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kAnchorThreads)
-anchor_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, double* __restrict__ inv_norm) {
-  dep_release();
-  const int b = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
-  if (r >= T) return;
-  const int vecs = D >> 3;
-  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(r) * D);
-  double n2a = 0.0, n2b = 0.0;
-  for (int v0 = lane; v0 < vecs; v0 += 128) {
-    uint4 q[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
-        n2a = fma(x0, x0, n2a);
-        n2b = fma(x1, x1, n2b);
-      }
-    }
-  }
-  const double n2 = warp_sum(n2a + n2b);
-  if (lane == 0) inv_norm[static_cast<int64_t>(b) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
-}
-
-// Per-head keys: the same pass over whole rows (all heads of a token are one contiguous row), with the sums taken per
-// 128-column block.  A warp covers 256 columns = two heads per step; lanes 0-15 reduce one head, lanes 16-31 the other.
-// Problem index of (chunk, head) = chunk * n_heads + head, as everywhere in the per-head path.
 __device__ __forceinline__ double half_warp_sum(double v) {
 #pragma unroll
   for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -115,123 +76,290 @@ __device__ __forceinline__ float half_warp_sum(float v) {
   return v;
 }
 
-__global__ void __launch_bounds__(kAnchorThreads)
-head_norms(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int H, double* __restrict__ inv_norm) {
-  dep_release();
-  const int chunk = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int r = blockIdx.x * (kAnchorThreads / 32) + warp;
-  if (r >= T) return;
-  const int vecs = D >> 3;
-  const uint4* row = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(r) * D);
-  for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
-    uint4 q[4];
-#pragma unroll
-    for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-      double n2a = 0.0, n2b = 0.0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const double x0 = bf16_to_f64(w[e] & 0xFFFFu), x1 = bf16_to_f64(w[e] >> 16);
-        n2a = fma(x0, x0, n2a);
-        n2b = fma(x1, x1, n2b);
-      }
-      const double n2 = half_warp_sum(n2a + n2b);
-      const int head = (v0 + 32 * u) >> 4;
-      if ((lane & 15) == 0 && head < H)
-        inv_norm[(static_cast<int64_t>(chunk) * H + head) * T + r] = n2 > 0.0 ? 1.0 / sqrt(n2) : 0.0;   // zero key: cosine 0
-    }
-  }
+// bf16 -> fp64 on the integer pipe, for NORMAL numbers: the double has the same sign, the exponent re-biased by
+// 1023 - 127 = 896 and the seven mantissa bits at the top of the fraction -- two or three integer operations where the
+// conversion instruction runs at a quarter of the fp64 multiply-add rate.  w holds two bf16 values (low and high half).
+// An exponent field of 0 (zero, subnormal) comes out as a number below 2^-126 and a field of 255 (Inf, NaN) as one of at
+// least 2^128: anchor_pass looks at every row's squared norm, and a group of rows with a norm outside [2^-40, 2^125] is
+// redone with the exact conversions below.  Inside that range a mis-read zero or subnormal moves a column sum by less
+// than 2^-126 * 2^40 = 2^-86 per row, far below the rounding of the fp64 sums themselves.
+__device__ __forceinline__ double bf16_lo_abs_fast(uint32_t w) {
+  return __hiloint2double(static_cast<int>(((w & 0x7FFFu) << 13) + 0x38000000u), 0);
+}
+__device__ __forceinline__ double bf16_hi_abs_fast(uint32_t w) {
+  return __hiloint2double(static_cast<int>(__umulhi(w & 0x7FFF0000u, 0x20000000u) + 0x38000000u), 0);
+}
+__device__ __forceinline__ double bf16_lo_fast(uint32_t w) {
+  return __hiloint2double(static_cast<int>((((w & 0x7FFFu) << 13) + 0x38000000u) | ((w << 16) & 0x80000000u)), 0);
+}
+__device__ __forceinline__ double bf16_hi_fast(uint32_t w) {
+  return __hiloint2double(static_cast<int>((__umulhi(w & 0x7FFF0000u, 0x20000000u) + 0x38000000u) | (w & 0x80000000u)), 0);
+}
+template <bool kExact> __device__ __forceinline__ double bf16_lo(uint32_t w) {
+  return kExact ? static_cast<double>(__uint_as_float(w << 16)) : bf16_lo_fast(w);
+}
+template <bool kExact> __device__ __forceinline__ double bf16_hi(uint32_t w) {
+  return kExact ? static_cast<double>(__uint_as_float(w & 0xFFFF0000u)) : bf16_hi_fast(w);
+}
+template <bool kExact> __device__ __forceinline__ double bf16_lo_abs(uint32_t w) {
+  return kExact ? static_cast<double>(__uint_as_float(w << 16)) : bf16_lo_abs_fast(w);
+}
+template <bool kExact> __device__ __forceinline__ double bf16_hi_abs(uint32_t w) {
+  return kExact ? static_cast<double>(__uint_as_float(w & 0xFFFF0000u)) : bf16_hi_abs_fast(w);
 }
 
-template <bool kPerHead>
-__global__ void __launch_bounds__(512)
-anchor_accumulate(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int D, int parts,
-                  const double* __restrict__ inv_norm, double* __restrict__ partial) {
-  dep_wait();
-  dep_release();
-  const int b = blockIdx.y, part = blockIdx.x / kColSplit, csplit = blockIdx.x % kColSplit;
-  const int tid = threadIdx.x, nthreads = blockDim.x;
-  const int vecs = D >> 3;
-  const int vec = csplit * nthreads + tid;   // the 16-byte column group this thread owns
-  // per-head keys: b is the chunk, the row is the whole token (D = all heads) and the norm is the one of this thread's head
-  const uint4* Kb = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * rm.stride);
-  const int rsv = D >> 3;   // row pitch in 16-byte vectors
-  const double* inv = inv_norm + (kPerHead ? (static_cast<int64_t>(b) * rm.hs + (vec >> 4)) : static_cast<int64_t>(b)) * T;
-  if (vec < vecs) {
-    double acc[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.0;
-    constexpr int U = 8;   // rows in flight per thread
-    for (int r0 = part; r0 < T; r0 += U * parts) {
-      uint4 q[U];
-      double sc[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int r = r0 + u * parts;
-        q[u] = r < T ? __ldg(Kb + static_cast<int64_t>(r) * rsv + vec) : make_uint4(0, 0, 0, 0);
-        sc[u] = r < T ? __ldg(inv + r) : 0.0;
+// ------------------------------------------------------------------------------------------------
+// anchor pass.  grid = (parts, chunks), 256 threads.  CTA (part, chunk) owns rows [part * rpp, (part + 1) * rpp) of
+// the chunk's anchor frame and walks them in groups of G rows:
+//   thread 0 keeps one bulk copy (the next group's G contiguous rows) in flight into the other half of the row buffer;
+//   phase 1: the 8 warps share the group's rows (8 / G column segments per row): fp64 squared norms from shared memory
+//            -> 1/|a| (0 for a zero key); with per-head keys (hs = n_heads) one norm per 128-column block, reduced
+//            within 16 lanes;
+//   phase 2: thread t owns the 16-byte column groups t, t + 256, ...: a_i[c] / |a_i| is added over the rows of the group.
+// The CTA writes its column sums as one slice; the last CTA of the chunk adds the slices in slice order and writes
+// m64, m32 = fp32(m64) and |m|^2 (per head with per-head keys).  VPT = 16-byte column groups per thread = ceil(D / 2048).
+// ------------------------------------------------------------------------------------------------
+constexpr int kAnchorThreads = 256;
+constexpr int kAnchorWarps = kAnchorThreads / 32;
+constexpr double kNorm2Lo = 8.2718061255302767e-25;    // 2^-80: squared norm below which a row is redone exactly
+constexpr double kNorm2Hi = 1.8092513943330656e+75;    // 2^250: likewise above
+
+// squared norms of the group's rows: warp -> (row, column segment); n2_s[row][seg] (whole keys) or n2_s[row][head]
+template <bool kExact>
+__device__ __forceinline__ void group_norms(const uint8_t* buf, size_t row_bytes, int rows, int nseg, int seg_vecs, int vecs,
+                                            int hs, int n2_pitch, double* n2_s) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int r = warp / nseg, seg = warp - r * nseg;
+  if (r >= rows) return;
+  const uint4* row = reinterpret_cast<const uint4*>(buf + r * row_bytes);
+  const int v_begin = seg * seg_vecs, v_end = min(vecs, v_begin + seg_vecs);
+  if (hs == 1) {
+    double n2a = 0.0, n2b = 0.0;
+    for (int v = v_begin + lane; v < v_end; v += 32) {
+      const uint4 q = row[v];
+      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+      // three of the eight conversions go to the conversion unit, five to the integer pipe: both stay busy
+      {
+        const double x0 = bf16_lo_abs<true>(w[0]), x1 = bf16_hi_abs<kExact>(w[0]);
+        const double x2 = bf16_lo_abs<kExact>(w[1]), x3 = bf16_hi_abs<true>(w[1]);
+        const double x4 = bf16_lo_abs<kExact>(w[2]), x5 = bf16_hi_abs<kExact>(w[2]);
+        const double x6 = bf16_lo_abs<true>(w[3]), x7 = bf16_hi_abs<kExact>(w[3]);
+        n2a = fma(x0, x0, n2a); n2b = fma(x1, x1, n2b);
+        n2a = fma(x2, x2, n2a); n2b = fma(x3, x3, n2b);
+        n2a = fma(x4, x4, n2a); n2b = fma(x5, x5, n2b);
+        n2a = fma(x6, x6, n2a); n2b = fma(x7, x7, n2b);
       }
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          acc[2 * e] = fma(bf16_to_f64(w[e] & 0xFFFFu), sc[u], acc[2 * e]);
-          acc[2 * e + 1] = fma(bf16_to_f64(w[e] >> 16), sc[u], acc[2 * e + 1]);
+    }
+    const double n2 = warp_sum(n2a + n2b);
+    if (lane == 0) n2_s[r * n2_pitch + seg] = n2;
+  } else {
+    for (int v = v_begin + lane; v - lane < v_end; v += 32) {   // a 32-lane step covers two heads: lanes 0-15 / 16-31
+      double n2a = 0.0, n2b = 0.0;
+      if (v < v_end) {
+        const uint4 q = row[v];
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+        {
+          const double x0 = bf16_lo_abs<true>(w[0]), x1 = bf16_hi_abs<kExact>(w[0]);
+          const double x2 = bf16_lo_abs<kExact>(w[1]), x3 = bf16_hi_abs<true>(w[1]);
+          const double x4 = bf16_lo_abs<kExact>(w[2]), x5 = bf16_hi_abs<kExact>(w[2]);
+          const double x6 = bf16_lo_abs<true>(w[3]), x7 = bf16_hi_abs<kExact>(w[3]);
+          n2a = fma(x0, x0, n2a); n2b = fma(x1, x1, n2b);
+          n2a = fma(x2, x2, n2a); n2b = fma(x3, x3, n2b);
+          n2a = fma(x4, x4, n2a); n2b = fma(x5, x5, n2b);
+          n2a = fma(x6, x6, n2a); n2b = fma(x7, x7, n2b);
         }
       }
+      const double n2 = half_warp_sum(n2a + n2b);
+      if ((lane & 15) == 0 && v < v_end) n2_s[r * n2_pitch + (v >> 4)] = n2;
     }
-    double* my = partial + (static_cast<int64_t>(b) * parts + part) * D + 8 * vec;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) my[e] = acc[e];
   }
 }
 
-// Adds the row slices of every problem in a fixed order: m64, m32 = fp32(m64) and this CTA's share of |m|^2.
-// grid = (ceil(D / 512), batch), 256 threads, two columns per thread; all loads are issued before the first addition.
-template <bool kPerHead>
-__global__ void __launch_bounds__(256)
-anchor_reduce(const double* __restrict__ partial, int T, int D, int parts, int H, double* __restrict__ m64,
-              float* __restrict__ m32, double* __restrict__ mnorm2_part) {
-  __shared__ double red2[8];
-  dep_wait();
-  dep_release();
-  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int c = 2 * (blockIdx.x * 256 + tid);
-  const double* pb = partial + static_cast<int64_t>(b) * parts * D;
-  double nn = 0.0;
-  if (c < D) {
-    double2 v[kMaxAnchorParts];
+// column sums of a / |a| over the rows of the group, for the 16-byte column groups this thread owns (t, t + 256, ...)
+template <int VPT, bool kExact>
+__device__ __forceinline__ void group_accumulate(const uint8_t* buf, size_t row_bytes, int rows, int vecs, int hs,
+                                                 const double* inv_s, double (&acc)[8 * VPT]) {
+  const int tid = threadIdx.x;
+  for (int r = 0; r < rows; ++r) {
+    const uint4* row = reinterpret_cast<const uint4*>(buf + r * row_bytes);
+    const double* inv = inv_s + r * hs;
 #pragma unroll
-    for (int p = 0; p < kMaxAnchorParts; ++p)
-      v[p] = p < parts ? __ldcg(reinterpret_cast<const double2*>(pb + static_cast<int64_t>(p) * D + c)) : make_double2(0.0, 0.0);
-    double t0 = 0.0, t1 = 0.0;
-#pragma unroll
-    for (int p = 0; p < kMaxAnchorParts; ++p) {
-      t0 += v[p].x;
-      t1 += v[p].y;
+    for (int i = 0; i < VPT; ++i) {
+      const int vec = tid + i * kAnchorThreads;
+      if (vec < vecs) {
+        const uint4 q = row[vec];
+        const double sc = inv[hs == 1 ? 0 : (vec >> 4)];
+        double* a = acc + 8 * i;
+        a[0] = fma(bf16_lo<true>(q.x), sc, a[0]);
+        a[1] = fma(bf16_hi<kExact>(q.x), sc, a[1]);
+        a[2] = fma(bf16_lo<kExact>(q.y), sc, a[2]);
+        a[3] = fma(bf16_hi<true>(q.y), sc, a[3]);
+        a[4] = fma(bf16_lo<kExact>(q.z), sc, a[4]);
+        a[5] = fma(bf16_hi<kExact>(q.z), sc, a[5]);
+        a[6] = fma(bf16_lo<true>(q.w), sc, a[6]);
+        a[7] = fma(bf16_hi<kExact>(q.w), sc, a[7]);
+      }
     }
-    t0 /= static_cast<double>(T);
-    t1 /= static_cast<double>(T);
-    *reinterpret_cast<double2*>(m64 + static_cast<int64_t>(b) * D + c) = make_double2(t0, t1);
-    *reinterpret_cast<float2*>(m32 + static_cast<int64_t>(b) * D + c) = make_float2(static_cast<float>(t0), static_cast<float>(t1));
-    nn = fma(t0, t0, fma(t1, t1, 0.0));
   }
-  nn = warp_sum(nn);
-  if (lane == 0) red2[warp] = nn;
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kAnchorThreads, VPT == 1 ? 4 : (VPT == 2 ? 3 : 2))
+anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int hs, int G, int rpp,
+            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
+            float* __restrict__ m32, double* __restrict__ mnorm2, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bar[2];
+  __shared__ uint32_t s_flag;
+  __shared__ double red[kAnchorWarps];
+  dep_release();
+  const int b = blockIdx.y, part = blockIdx.x, parts = gridDim.x;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const size_t row_bytes = static_cast<size_t>(D) * 2;
+  const int nseg = kAnchorWarps / G;                                        // column segments per row in phase 1
+  const int n2_pitch = hs == 1 ? nseg : hs;
+  uint8_t* rows_s = smem;                                                   // [2][G][D] bf16
+  double* inv_s = reinterpret_cast<double*>(smem + 2 * G * row_bytes);      // [G][hs]
+  double* n2_s = inv_s + G * hs;                                            // [G][n2_pitch]
+  const int r0 = min(T, part * rpp), r1 = min(T, r0 + rpp);
+  const int n_groups = (r1 - r0 + G - 1) / G;
+  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride;
+  if (tid == 0) {
+    ptx::mbar_init(&bar[0], 1);
+    ptx::mbar_init(&bar[1], 1);
+    ptx::fence_mbar_init();
+  }
   __syncthreads();
-  if (kPerHead) {
-    // a warp covers 64 columns: two warps per head, four heads per block; |m_h|^2 is one share per (chunk, head)
-    const int head = blockIdx.x * 4 + tid;
-    if (tid < 4 && head < H)
-      mnorm2_part[(static_cast<int64_t>(b) * H + head) * kMaxNormParts] = red2[2 * tid] + red2[2 * tid + 1];
-  } else if (tid == 0) {
-    double t = 0.0;
-    for (int w = 0; w < 8; ++w) t += red2[w];
-    mnorm2_part[static_cast<int64_t>(b) * kMaxNormParts + blockIdx.x] = t;
+  auto issue = [&](int g) {   // thread 0: one bulk copy of the group's rows (contiguous in memory)
+    const int ra = r0 + g * G;
+    const uint32_t bytes = static_cast<uint32_t>(min(G, r1 - ra) * row_bytes);
+    ptx::mbar_expect_tx(&bar[g & 1], bytes);
+    ptx::bulk_load_1d(rows_s + (g & 1) * G * row_bytes, Kb + static_cast<int64_t>(ra) * D, bytes, &bar[g & 1]);
+  };
+  if (tid == 0 && n_groups > 0) issue(0);
+  double acc[8 * VPT];
+#pragma unroll
+  for (int i = 0; i < 8 * VPT; ++i) acc[i] = 0.0;
+  const int vecs = D >> 3;
+  const int seg_vecs = (((vecs >> 4) + nseg - 1) / nseg) << 4;   // whole 128-column blocks per segment
+  int armed = n_groups > 0 ? 1 : 0;   // groups whose copy has been issued
+  int g = 0;
+  for (; g < n_groups; ++g) {
+    if (g + 1 < n_groups) {
+      if (tid == 0) issue(g + 1);     // its buffer was released by the barrier that ended group g - 1
+      armed = g + 2;
+    }
+    const bool landed = ptx::mbar_wait(&bar[g & 1], (g >> 1) & 1);
+    if (__syncthreads_or(!landed)) {  // a copy that never lands: report, stop reading, still hand in the slice
+      if (tid == 0) atomicOr(status, WK_DEV_TIMEOUT);
+      break;
+    }
+    const int rows = min(G, r1 - (r0 + g * G));
+    const uint8_t* buf = rows_s + (g & 1) * G * row_bytes;
+    // ---- phase 1: norms (integer-pipe conversions; redone exactly when a norm falls outside the safe range)
+    group_norms<false>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
+    __syncthreads();
+    bool redo = false;
+    auto finish_norms = [&](bool check) {
+      for (int i = tid; i < rows * hs; i += kAnchorThreads) {
+        const int r = i / hs, h = i - r * hs;
+        double n2 = 0.0;
+        if (hs == 1) for (int sg = 0; sg < nseg; ++sg) n2 += n2_s[r * n2_pitch + sg];
+        else n2 = n2_s[r * n2_pitch + h];
+        inv_s[i] = n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);   // zero key: cosine 0; a NaN norm stays NaN
+        if (check) redo = redo || !(n2 >= kNorm2Lo && n2 <= kNorm2Hi);
+      }
+    };
+    finish_norms(true);
+    const bool exact = __syncthreads_or(redo) != 0;
+    if (exact) {
+      group_norms<true>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
+      __syncthreads();
+      finish_norms(false);
+      __syncthreads();
+      group_accumulate<VPT, true>(buf, row_bytes, rows, vecs, hs, inv_s, acc);
+    } else {
+      // ---- phase 2
+      group_accumulate<VPT, false>(buf, row_bytes, rows, vecs, hs, inv_s, acc);
+    }
+    __syncthreads();   // the group's buffer, inv_s and n2_s may be overwritten from here on
   }
+  // a copy still in flight when the loop was left early must land before the CTA gives up its shared memory
+  if (tid == 0) {
+    for (int gg = g; gg < armed; ++gg)   // empty unless the loop was left at group g < n_groups
+      for (uint32_t i = 0; i < (1u << 16); ++i)
+        if (ptx::mbar_try_wait(&bar[gg & 1], (gg >> 1) & 1)) break;
+  }
+  // ---- this CTA's slice
+  double* my = partial + (static_cast<int64_t>(b) * max_parts + part) * D;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vec = tid + i * kAnchorThreads;
+    if (vec < vecs) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        __stcg(reinterpret_cast<double2*>(my + 8 * vec) + e, make_double2(acc[8 * i + 2 * e], acc[8 * i + 2 * e + 1]));
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_flag = (atomicAdd(&tickets[b], 1u) == static_cast<uint32_t>(parts - 1)) ? 1u : 0u;
+  __syncthreads();
+  if (!s_flag) return;
+  // ---- last CTA of the chunk: add the slices in slice order.  Thread t owns column pairs t, t + 256, ...; eight
+  // slices' worth of loads are in flight before the first addition.
+  __threadfence();
+  const double* pb = partial + static_cast<int64_t>(b) * max_parts * D;
+  const double inv_T = 1.0 / static_cast<double>(T);
+  const int pairs = D >> 1;
+  double nn_all = 0.0;
+  for (int c0 = 0; c0 < pairs; c0 += kAnchorThreads) {   // uniform trip count: the per-head sums use block barriers
+    const int c = c0 + tid;
+    double t0 = 0.0, t1 = 0.0;
+    if (c < pairs) {
+      for (int p0 = 0; p0 < parts; p0 += 8) {
+        double2 v[8];
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp)
+          v[pp] = p0 + pp < parts ? __ldcg(reinterpret_cast<const double2*>(pb + static_cast<int64_t>(p0 + pp) * D) + c)
+                                  : make_double2(0.0, 0.0);
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp) {
+          t0 += v[pp].x;
+          t1 += v[pp].y;
+        }
+      }
+      t0 *= inv_T;
+      t1 *= inv_T;
+      reinterpret_cast<double2*>(m64 + static_cast<int64_t>(b) * D)[c] = make_double2(t0, t1);
+      reinterpret_cast<float2*>(m32 + static_cast<int64_t>(b) * D)[c] =
+          make_float2(static_cast<float>(t0), static_cast<float>(t1));
+    }
+    const double nn = fma(t0, t0, t1 * t1);
+    if (hs == 1) {
+      nn_all += nn;
+    } else {
+      // 64 column pairs per head: warps 2j and 2j + 1 of this step hold head c0 / 64 + j
+      const double wsum = warp_sum(nn);
+      __syncthreads();
+      if (lane == 0) red[warp] = wsum;
+      __syncthreads();
+      const int head = (c0 >> 6) + tid;
+      if (tid < kAnchorWarps / 2 && head < hs)
+        mnorm2[(static_cast<int64_t>(b) * hs + head) * kMaxNormParts] = red[2 * tid] + red[2 * tid + 1];
+    }
+  }
+  if (hs == 1) {
+    const double wsum = warp_sum(nn_all);
+    if (lane == 0) red[warp] = wsum;
+    __syncthreads();
+    if (tid == 0) {
+      double t = 0.0;
+      for (int w = 0; w < kAnchorWarps; ++w) t += red[w];
+      mnorm2[static_cast<int64_t>(b) * kMaxNormParts] = t;
+    }
+  }
+  if (tid == 0) tickets[b] = 0;   // ready for the next call
 }
 
 // Fallback for very wide rows (D > 8192): same arithmetic, accumulators in shared memory.
@@ -299,133 +427,8 @@ anchor_pass_wide(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int
 }
 
 // ------------------------------------------------------------------------------------------------
-// score pass.  grid = (ceil(NA / kScoreRowsPerCta), batch); one warp per row; m32 staged in shared memory.
-// Per lane the fp32 accumulation is a chain of 8 * ceil(D/256) fused multiply-adds followed by five
-// shuffle additions; select_pass derives its error band from exactly this order.
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kScoreThreads)
-score_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D,
-           const float* __restrict__ m32, float* __restrict__ s32, float* __restrict__ scores_out,
-           uint32_t* __restrict__ status) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  dep_wait();
-  dep_release();
-  float4* m = reinterpret_cast<float4*>(smem);   // [D/4]
-  const int b = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
-  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
-  __syncthreads();
-  const int vecs = D >> 3;
-  const int j0 = blockIdx.x * kScoreRowsPerCta;
-  const int j1 = min(NA, j0 + kScoreRowsPerCta);
-  const int pitch = D;
-  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * pitch;
-  // two rows per warp at a time, so that twice as many 16-byte loads are in flight
-  constexpr int W = kScoreThreads / 32;
-  for (int j = j0 + warp; j < j1; j += 2 * W) {
-    const int jb = j + W;
-    const bool has_b = jb < j1;
-    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * pitch);
-    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * pitch);
-    float dot_a = 0.f, n2_a = 0.f, dot_b = 0.f, n2_b = 0.f;
-    for (int v0 = lane; v0 < vecs; v0 += 128) {
-      uint4 qa[4], qb[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int v = v0 + 32 * u;
-        qa[u] = v < vecs ? __ldg(row_a + v) : make_uint4(0, 0, 0, 0);
-        qb[u] = v < vecs ? __ldg(row_b + v) : make_uint4(0, 0, 0, 0);
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int v = v0 + 32 * u;
-        if (v < vecs) {
-          const float4 ma = m[2 * v], mb = m[2 * v + 1];
-          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-          const uint32_t wa[4] = {qa[u].x, qa[u].y, qa[u].z, qa[u].w}, wb[4] = {qb[u].x, qb[u].y, qb[u].z, qb[u].w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float x;
-            x = bf16lo(wa[e]); dot_a = fmaf(x, mm[2 * e], dot_a); n2_a = fmaf(x, x, n2_a);
-            x = bf16hi(wa[e]); dot_a = fmaf(x, mm[2 * e + 1], dot_a); n2_a = fmaf(x, x, n2_a);
-            x = bf16lo(wb[e]); dot_b = fmaf(x, mm[2 * e], dot_b); n2_b = fmaf(x, x, n2_b);
-            x = bf16hi(wb[e]); dot_b = fmaf(x, mm[2 * e + 1], dot_b); n2_b = fmaf(x, x, n2_b);
-          }
-        }
-      }
-    }
-    dot_a = warp_sum(dot_a);
-    n2_a = warp_sum(n2_a);
-    dot_b = warp_sum(dot_b);
-    n2_b = warp_sum(n2_b);
-    if (lane < 2 && (lane == 0 || has_b)) {
-      const float dot = lane ? dot_b : dot_a, n2 = lane ? n2_b : n2_a;
-      const int jj = lane ? jb : j;
-      const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
-      if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
-      s32[static_cast<int64_t>(b) * NA + jj] = sc;
-      if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
-    }
-  }
-}
-
-// Per-head keys: whole rows again, the dot product and the squared norm taken per 128-column block (lanes 0-15 / 16-31
-// of a 256-column step).  Per lane and head: 8 fused multiply-adds, then 4 shuffle additions -- inside the error band
-// select_pass derives for D = 128.
-__global__ void __launch_bounds__(kScoreThreads)
-head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int H, const float* __restrict__ m32,
-           float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  dep_wait();
-  dep_release();
-  float4* m = reinterpret_cast<float4*>(smem);   // [D/4]: the heads' mean unit anchors, side by side
-  const int chunk = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(chunk) * D);
-  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
-  __syncthreads();
-  const int vecs = D >> 3;
-  const int j0 = blockIdx.x * kScoreRowsPerCta;
-  const int j1 = min(NA, j0 + kScoreRowsPerCta);
-  const __nv_bfloat16* Kb = K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(T) * D;
-  constexpr int W = kScoreThreads / 32;
-  for (int j = j0 + warp; j < j1; j += W) {
-    const uint4* row = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
-    for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
-      uint4 q[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int v = v0 + 32 * u;
-        float dot = 0.f, n2 = 0.f;
-        if (v < vecs) {
-          const float4 ma = m[2 * v], mb = m[2 * v + 1];
-          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float x;
-            x = bf16lo(w[e]); dot = fmaf(x, mm[2 * e], dot); n2 = fmaf(x, x, n2);
-            x = bf16hi(w[e]); dot = fmaf(x, mm[2 * e + 1], dot); n2 = fmaf(x, x, n2);
-          }
-        }
-        dot = half_warp_sum(dot);
-        n2 = half_warp_sum(n2);
-        const int head = v >> 4;
-        if ((lane & 15) == 0 && head < H) {
-          const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
-          if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
-          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + j;
-          s32[at] = sc;
-          if (scores_out) scores_out[at] = sc;
-        }
-      }
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
-// select pass.  One CTA per problem.
+// selection of one problem by one CTA of kThr threads (a device function: the score kernel's last CTA of a problem calls
+// it in place; per-head keys and the trivial cases n_keep = 0 / all have a kernel of their own around it).
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t f32_key(float f) {   // order-preserving map float -> uint32
   uint32_t u = __float_as_uint(f);
@@ -435,15 +438,11 @@ __device__ __forceinline__ float key_f32(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-template <bool kPerHead>
-__global__ void __launch_bounds__(kPerHead ? kSelectThreadsHead : kSelectThreads)
-select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D, int n_keep,
-            const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
-            int n_norm_parts, int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  // a problem of 128 columns has little to do in the refinement: a quarter of the threads, four problems per SM at once
-  constexpr int kThr = kPerHead ? kSelectThreadsHead : kSelectThreads;
-  dep_wait();
+template <int kThr, bool kPerHead>
+__device__ __forceinline__ void select_problem(uint8_t* smem, int b, const __nv_bfloat16* __restrict__ K, RowMap rm, int T,
+                                               int NA, int D, int n_keep, const float* __restrict__ s32,
+                                               const double* __restrict__ m64, const double* __restrict__ mnorm,
+                                               int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem);                       // [NA]
   int32_t* band_idx = reinterpret_cast<int32_t*>(keys + NA);                // [NA]
   double* band_s = reinterpret_cast<double*>(band_idx + NA);                // [NA] (8-byte aligned: 8*NA)
@@ -452,7 +451,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   __shared__ uint32_t sel_prefix, sel_rank, n_band, n_below;
   __shared__ uint32_t warp_tot[32];
   __shared__ double band_red[8][kThr / 32];
-  const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int C = T + n_keep;
   int32_t* out = keep_idx + static_cast<int64_t>(b) * C;
   for (int i = tid; i < T; i += kThr) out[i] = i;                 // the anchor frame is kept whole
@@ -462,7 +461,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
     return;
   }
   const float* sb = s32 + static_cast<int64_t>(b) * NA;
-  for (int j = tid; j < NA; j += kThr) keys[j] = f32_key(sb[j]);
+  for (int j = tid; j < NA; j += kThr) keys[j] = f32_key(__ldcg(sb + j));   // written by other CTAs: read through L2
   if (tid == 0) { sel_prefix = 0; sel_rank = static_cast<uint32_t>(n_keep - 1); n_band = 0; n_below = 0; }
   __syncthreads();
   // radix select: the key of 0-based rank n_keep-1
@@ -506,8 +505,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   // fp32 error band.  Per lane: n_l = 8*ceil(D/256) products in a fused chain, then 5 shuffle adds, the rounding of
   // m to fp32, the norm (same chain), one sqrt and one division: |s32 - s| <= (2 n_l + 32) 2^-24 |m|.
   const int n_l = 8 * ((D + 255) / 256);
-  double mn2 = 0.0;
-  for (int i = 0; i < n_norm_parts; ++i) mn2 += mnorm[static_cast<int64_t>(b) * kMaxNormParts + i];
+  const double mn2 = __ldcg(mnorm + static_cast<int64_t>(b) * kMaxNormParts);
   const double eps = (2.0 * n_l + 32.0) * 5.9604644775390625e-08 * sqrt(mn2) * 1.000001;
   const double lo = static_cast<double>(theta) - 2.0 * eps;
   const double hi = static_cast<double>(theta) + 2.0 * eps;
@@ -622,6 +620,185 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
   }
 }
 
+// One CTA per problem: per-head keys (n_heads problems per chunk) and the cases that need no scores.
+constexpr int kSelectThreads = 256;
+template <bool kPerHead>
+__global__ void __launch_bounds__(kSelectThreads)
+select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D, int n_keep,
+            const float* __restrict__ s32, const double* __restrict__ m64, const double* __restrict__ mnorm,
+            int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
+  select_problem<kSelectThreads, kPerHead>(smem, blockIdx.x, K, rm, T, NA, D, n_keep, s32, m64, mnorm, keep_idx, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// score pass + selection.  grid = blocks of kScoreRowsPerCta rows, problem-major (blockIdx.x = b * nblk + block), so that
+// the problems finish in order; one warp per row; m32 staged in shared memory.  The CTA that hands in the last rows of
+// a problem (atomic ticket; nobody waits) runs that problem's selection on the spot, under the streaming of the
+// problems behind it.
+// Per lane the fp32 accumulation is two chains of 4 * ceil(D/256) fused multiply-adds (the low and the high halves of
+// the packed pairs), one addition of the two, then five shuffle additions: no deeper than the single chain of
+// 8 * ceil(D/256) + 5 operations the selection's error band is derived for.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kScoreThreads)
+score_select(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int n_keep, int nblk,
+             const float* __restrict__ m32, const double* __restrict__ m64, const double* __restrict__ mnorm,
+             float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ tickets,
+             int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  __shared__ uint32_t s_last;
+  dep_wait();
+  dep_release();
+  float4* m = reinterpret_cast<float4*>(smem);   // [D/4]; the selection reuses the space afterwards
+  const int b = blockIdx.x / nblk, blk = blockIdx.x - b * nblk;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
+  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
+  __syncthreads();
+  const int vecs = D >> 3;
+  const int j0 = blk * kScoreRowsPerCta;
+  const int j1 = min(NA, j0 + kScoreRowsPerCta);
+  const int pitch = D;
+  const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * pitch;
+  // two rows per warp at a time, so that twice as many 16-byte loads are in flight
+  constexpr int W = kScoreThreads / 32;
+  for (int j = j0 + warp; j < j1; j += 2 * W) {
+    const int jb = j + W;
+    const bool has_b = jb < j1;
+    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * pitch);
+    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * pitch);
+    // packed fp32 pairs: one instruction multiplies-and-adds the two bf16 values of a 32-bit word; the low and the high
+    // halves keep separate sums (half as long as a single chain would be), added once at the end
+    uint64_t dot2_a = 0, n22_a = 0, dot2_b = 0, n22_b = 0;
+    for (int v0 = lane; v0 < vecs; v0 += 128) {
+      uint4 qa[4], qb[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u;
+        qa[u] = v < vecs ? __ldg(row_a + v) : make_uint4(0, 0, 0, 0);
+        qb[u] = v < vecs ? __ldg(row_b + v) : make_uint4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u;
+        if (v < vecs) {
+          const float4 ma = m[2 * v], mb = m[2 * v + 1];
+          const uint64_t mm[4] = {ptx::pack_f32x2(ma.x, ma.y), ptx::pack_f32x2(ma.z, ma.w), ptx::pack_f32x2(mb.x, mb.y),
+                                  ptx::pack_f32x2(mb.z, mb.w)};
+          const uint32_t wa[4] = {qa[u].x, qa[u].y, qa[u].z, qa[u].w}, wb[4] = {qb[u].x, qb[u].y, qb[u].z, qb[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const uint64_t xa = ptx::pack_f32x2(bf16lo(wa[e]), bf16hi(wa[e]));
+            const uint64_t xb = ptx::pack_f32x2(bf16lo(wb[e]), bf16hi(wb[e]));
+            dot2_a = ptx::fma_f32x2(xa, mm[e], dot2_a);
+            n22_a = ptx::fma_f32x2(xa, xa, n22_a);
+            dot2_b = ptx::fma_f32x2(xb, mm[e], dot2_b);
+            n22_b = ptx::fma_f32x2(xb, xb, n22_b);
+          }
+        }
+      }
+    }
+    float lo_, hi_;
+    ptx::unpack_f32x2(dot2_a, lo_, hi_); float dot_a = lo_ + hi_;
+    ptx::unpack_f32x2(n22_a, lo_, hi_);  float n2_a = lo_ + hi_;
+    ptx::unpack_f32x2(dot2_b, lo_, hi_); float dot_b = lo_ + hi_;
+    ptx::unpack_f32x2(n22_b, lo_, hi_);  float n2_b = lo_ + hi_;
+    dot_a = warp_sum(dot_a);
+    n2_a = warp_sum(n2_a);
+    dot_b = warp_sum(dot_b);
+    n2_b = warp_sum(n2_b);
+    if (lane < 2 && (lane == 0 || has_b)) {
+      const float dot = lane ? dot_b : dot_a, n2 = lane ? n2_b : n2_a;
+      const int jj = lane ? jb : j;
+      const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
+      if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+      s32[static_cast<int64_t>(b) * NA + jj] = sc;
+      if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
+    }
+  }
+  if (keep_idx == nullptr) return;   // scores only
+  // hand in this block of rows; the CTA that completes the problem selects
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&tickets[b], 1u) == static_cast<uint32_t>(nblk - 1)) ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (tid == 0) tickets[b] = 0;   // ready for the next call
+  const RowMap rm{stride, D, 1};
+  select_problem<kScoreThreads, false>(smem, b, K, rm, T, NA, D, n_keep, s32, m64, mnorm, keep_idx, status);
+}
+
+// Per-head keys: whole rows again, the dot product and the squared norm taken per 128-column block (lanes 0-15 / 16-31
+// of a 256-column step).  Per lane and head: 8 fused multiply-adds, then 4 shuffle additions -- inside the error band
+// select_pass derives for D = 128.
+__global__ void __launch_bounds__(kScoreThreads)
+head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int H, const float* __restrict__ m32,
+           float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
+  dep_release();
+  float4* m = reinterpret_cast<float4*>(smem);   // [D/4]: the heads' mean unit anchors, side by side
+  const int chunk = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(chunk) * D);
+  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
+  __syncthreads();
+  const int vecs = D >> 3;
+  const int j0 = blockIdx.x * kScoreRowsPerCta;
+  const int j1 = min(NA, j0 + kScoreRowsPerCta);
+  const __nv_bfloat16* Kb = K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(T) * D;
+  constexpr int W = kScoreThreads / 32;
+  for (int j = j0 + warp; j < j1; j += W) {
+    const uint4* row = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
+    for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u;
+        float dot = 0.f, n2 = 0.f;
+        if (v < vecs) {
+          const float4 ma = m[2 * v], mb = m[2 * v + 1];
+          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
+          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float x;
+            x = bf16lo(w[e]); dot = fmaf(x, mm[2 * e], dot); n2 = fmaf(x, x, n2);
+            x = bf16hi(w[e]); dot = fmaf(x, mm[2 * e + 1], dot); n2 = fmaf(x, x, n2);
+          }
+        }
+        dot = half_warp_sum(dot);
+        n2 = half_warp_sum(n2);
+        const int head = v >> 4;
+        if ((lane & 15) == 0 && head < H) {
+          const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
+          if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + j;
+          s32[at] = sc;
+          if (scores_out) scores_out[at] = sc;
+        }
+      }
+    }
+  }
+}
+
+}  // namespace
+
+namespace {
+
+template <int VPT>
+void launch_anchor(dim3 grid, size_t smem, cudaStream_t s, const __nv_bfloat16* K, int64_t stride, int T, int D, int hs,
+                   int G, int rpp, double* partial, int max_parts, uint32_t* tickets, double* m64, float* m32,
+                   double* mnorm2, uint32_t* status) {
+  if (smem > 48 * 1024)
+    cudaFuncSetAttribute(anchor_pass<VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  anchor_pass<VPT><<<grid, kAnchorThreads, smem, s>>>(K, stride, T, D, hs, G, rpp, partial, max_parts, tickets, m64, m32,
+                                                      mnorm2, status);
+}
+
 }  // namespace
 
 wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int chunks, int32_t* keep_idx,
@@ -640,50 +817,73 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   float* s32 = reinterpret_cast<float*>(sc + ctx->sl.s32_off);
   double* mnorm = reinterpret_cast<double*>(sc + ctx->sl.mnorm_off);
   double* partial = reinterpret_cast<double*>(sc + ctx->sl.part_off);
-  uint32_t* counters = reinterpret_cast<uint32_t*>(sc + ctx->sl.cnt_off);
-  const int parts = ctx->sl.anchor_parts;
+  uint32_t* tickets = reinterpret_cast<uint32_t*>(sc + ctx->sl.cnt_off);   // [2][max_batch]: anchor pass, score pass
+  const int max_parts = ctx->sl.anchor_parts;
   const bool need_scores = (n_keep > 0 && n_keep < NA) || scores_out != nullptr;
+  const size_t smem_sel = static_cast<size_t>(NA) * (4 + 4 + 8 + 1) + 16;
+  const size_t smem_m = static_cast<size_t>(DF) * sizeof(float);
+  if (smem_sel > 200 * 1024 || smem_m > 200 * 1024) return WK_ERR_SHAPE;
   wk_status st = WK_OK;
-  int n_norm_parts = 1;
   if (need_scores) {
     if (DF <= 8192) {
-      n_norm_parts = per_head ? 1 : (DF + 511) / 512;
-      double* inv_norm = reinterpret_cast<double*>(sc + ctx->sl.inv_off);
-      const dim3 grid_n((T + kAnchorThreads / 32 - 1) / (kAnchorThreads / 32), chunks);
-      if (per_head) head_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, DF, H, inv_norm);
-      else anchor_norms<<<grid_n, kAnchorThreads, 0, s>>>(K, stride, T, DF, inv_norm);
-      if ((st = after_launch(ctx)) != WK_OK) return st;
-      const int threads = ((DF / 8 + kColSplit * 32 - 1) / (kColSplit * 32)) * 32;
-      const dim3 grid_acc(parts * kColSplit, chunks);
-      if (per_head) launch_chained(anchor_accumulate<true>, grid_acc, dim3(threads), 0, s, K, rm, T, DF, parts, inv_norm, partial);
-      else launch_chained(anchor_accumulate<false>, grid_acc, dim3(threads), 0, s, K, rm, T, DF, parts, inv_norm, partial);
-      if ((st = after_launch(ctx)) != WK_OK) return st;
-      const dim3 grid_r((DF + 511) / 512, chunks);
-      if (per_head) launch_chained(anchor_reduce<true>, grid_r, dim3(256), 0, s, partial, T, DF, parts, H, m64, m32, mnorm);
-      else launch_chained(anchor_reduce<false>, grid_r, dim3(256), 0, s, partial, T, DF, parts, H, m64, m32, mnorm);
+      // rows per group: two groups of G rows of DF bf16 in shared memory, at most one row per warp
+      int G = kAnchorWarps;
+      while (G > 1 && 2 * static_cast<size_t>(G) * DF * 2 > 100 * 1024) G >>= 1;
+      const int hs_a = per_head ? H : 1, nseg = kAnchorWarps / G;
+      const size_t smem_a = 2 * static_cast<size_t>(G) * DF * 2 +
+                            static_cast<size_t>(G) * (hs_a + (hs_a > nseg ? hs_a : nseg)) * sizeof(double);
+      // slices per chunk: as many CTAs as the machine holds at once, so that every SM carries the same number of them
+      // (a grid that leaves slots empty is spread unevenly: some SMs take their full share, others half of it)
+      int per_sm = static_cast<int>((220 * 1024) / (smem_a + 1024));
+      const int by_regs = DF > 2048 ? 2 : 4;
+      if (per_sm > by_regs) per_sm = by_regs;
+      int parts = ctx->sm_count * (per_sm < 1 ? 1 : per_sm) / chunks;
+      if (parts < 1) parts = 1;
+      if (parts > max_parts) parts = max_parts;
+      if (parts > (T + G - 1) / G) parts = (T + G - 1) / G;
+      int rpp = (T + parts - 1) / parts;
+      rpp = (rpp + G - 1) / G * G;            // whole groups, so that only a chunk's last slice has a short group
+      parts = (T + rpp - 1) / rpp;
+      const dim3 grid(parts, chunks);
+      const int hs = per_head ? H : 1;
+      const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 1 .. 4 for DF <= 8192
+#define WK_ANCHOR(V) launch_anchor<V>(grid, smem_a, s, K, stride, T, DF, hs, G, rpp, partial, max_parts, tickets, m64, m32, mnorm, ctx->status_dev)
+      if (vpt <= 1) WK_ANCHOR(1);
+      else if (vpt == 2) WK_ANCHOR(2);
+      else if (vpt == 3) WK_ANCHOR(3);
+      else WK_ANCHOR(4);
+#undef WK_ANCHOR
     } else {
       if (per_head) return WK_ERR_SHAPE;   // rows wider than 8,192 columns take the whole-key fallback only
-      const dim3 grid_a(parts, chunks);
+      const dim3 grid_a(max_parts, chunks);
       const size_t smem_acc = static_cast<size_t>(DF) * sizeof(double);
       if (smem_acc > 200 * 1024) return WK_ERR_SHAPE;
       WK_CUDA_TRY(ctx, cudaFuncSetAttribute(anchor_pass_wide, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             static_cast<int>(smem_acc)));
-      anchor_pass_wide<<<grid_a, kAnchorThreads, smem_acc, s>>>(K, stride, T, DF, parts, partial, counters, m64, m32,
+      anchor_pass_wide<<<grid_a, kAnchorThreads, smem_acc, s>>>(K, stride, T, DF, max_parts, partial, tickets, m64, m32,
                                                                 mnorm);
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
-    const dim3 grid_s((NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta, chunks);
-    const size_t smem_m = static_cast<size_t>(DF) * sizeof(float);
-    if (per_head)
-      launch_chained(head_score, grid_s, dim3(kScoreThreads), smem_m, s, K, stride, T, NA, DF, H, m32, s32, scores_out,
-                     ctx->status_dev);
-    else
-      launch_chained(score_pass, grid_s, dim3(kScoreThreads), smem_m, s, K, stride, T, NA, DF, m32, s32, scores_out,
-                     ctx->status_dev);
-    if ((st = after_launch(ctx)) != WK_OK) return st;
+    const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
+    if (per_head) {
+      if (smem_m > 48 * 1024)
+        WK_CUDA_TRY(ctx, cudaFuncSetAttribute(head_score, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_m)));
+      launch_chained(head_score, dim3(nblk, chunks), dim3(kScoreThreads), smem_m, s, K, stride, T, NA, DF, H, m32, s32,
+                     scores_out, ctx->status_dev);
+      if ((st = after_launch(ctx)) != WK_OK) return st;
+    } else {
+      const bool select_here = n_keep > 0 && n_keep < NA;
+      const size_t smem_s = select_here && smem_sel > smem_m ? smem_sel : smem_m;
+      if (smem_s > 48 * 1024)
+        WK_CUDA_TRY(ctx, cudaFuncSetAttribute(score_select, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_s)));
+      launch_chained(score_select, dim3(static_cast<unsigned>(nblk) * chunks), dim3(kScoreThreads), smem_s, s, K, stride, T, NA,
+                     DF, n_keep, nblk, m32, m64, mnorm, s32, scores_out, tickets + ctx->max_batch,
+                     select_here ? keep_idx : static_cast<int32_t*>(nullptr), ctx->status_dev);
+      if ((st = after_launch(ctx)) != WK_OK) return st;
+      if (select_here) return WK_OK;
+    }
   }
-  const size_t smem_sel = static_cast<size_t>(NA) * (4 + 4 + 8 + 1) + 16;
-  if (smem_sel > 200 * 1024) return WK_ERR_SHAPE;
+  // per-head keys, and the cases that need no scores (n_keep = 0 or everything kept): a selection launch of its own
   if (smem_sel > 48 * 1024) {
     WK_CUDA_TRY(ctx, cudaFuncSetAttribute(select_pass<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(smem_sel)));
@@ -691,11 +891,11 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
                                           static_cast<int>(smem_sel)));
   }
   if (per_head)
-    launch_chained(select_pass<true>, dim3(batch), dim3(kSelectThreadsHead), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
-                   n_norm_parts, keep_idx, ctx->status_dev);
+    launch_chained(select_pass<true>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
+                   keep_idx, ctx->status_dev);
   else
     launch_chained(select_pass<false>, dim3(batch), dim3(kSelectThreads), smem_sel, s, K, rm, T, NA, D, n_keep, s32, m64, mnorm,
-                   n_norm_parts, keep_idx, ctx->status_dev);
+                   keep_idx, ctx->status_dev);
   return after_launch(ctx);
 }
 
