@@ -1,21 +1,34 @@
 // World Retrieval (Eq. 4, distance of Section 5.1) over a pose array of any length: the same fp64 arithmetic and the
-// same tie rule as retrieve_kernel, organised as a streaming scan so that millions of candidates run at memory speed.
+// same tie rule as retrieve_kernel, organised so that millions of candidates are read from memory ONCE.
 //
-//   scan_init    resets the header (maxima, candidate count)
-//   scan_max     pass 1: max squared translation distance and min |quaternion dot| over the valid candidates
-//                (order-independent: integer atomics on the bit patterns of non-negative doubles)
-//   scan_select  pass 2: every block keeps the k best (distance, index) pairs of its share.  A candidate is dropped
-//                as soon as a lower bound of its distance exceeds the block's current k-th best, which spares most of
-//                them the divisions and the acos; survivors go to a shared-memory list that is cut back to k by exact
-//                rank counting whenever it fills
-//   scan_merge   one block repeats that selection over the blocks' lists and writes the result in rank order
+// The distance d_i = t_i / max t + r_i / max r needs both maxima, which are only known after every pose has been seen.
+// What can be decided earlier: if k real candidates ("pivots") are certain to be closer than candidate j whatever the
+// two maxima turn out to be, j is not among the k best.  With T* / R* the largest translation / rotation term of the
+// pivots, mt_lo any lower bound of max t, and max r <= pi (an angle), that holds when
+//       r_j > R* + (pi / mt_lo) * max(0, T* - t_j)
+// (a pivot with the larger translation term loses at most (T* - t_j) / mt_lo there and gains at least (r_j - R*) / pi).
 //
-// Nothing here depends on the order in which threads or blocks run: the k best under (distance, index) are unique.
+//   scan_sample  a strided sample of the candidates (one in 64, 2^15 .. 2^18 of them): per block the largest t,
+//                and for each of k disjoint sample classes the candidate with the smallest r + pi t / (roughly max t),
+//                in fp32 -- pivots only have to be real candidates, not the best ones
+//   scan_filter  the single pass over all poses: every block first merges the sample blocks' records and takes the
+//                pivots' exact fp64 terms (T*, R*, mt_lo); then per candidate a dozen fp32 operations: the test above
+//                with every quantity rounded to the safe side, and running fp32 maxima -- the exact fp64 terms are
+//                only formed for a candidate whose fp32 value comes within rounding of the thread's record, so the true
+//                maxima are never missed.  Survivors (typically 1-2 %) go to an index list
+//   scan_select  the exact distances of the listed candidates with the final maxima: every block keeps its k best by
+//                rank counting under (distance, index).  If the list overflowed (poses that cannot be pruned, e.g. all
+//                rotations equal) it walks all poses instead: the two-read path, slower but always right.  The block
+//                that hands in its list last (atomic ticket) merges the lists and writes the result in rank order
+//
+// Nothing here depends on the order in which threads or blocks run: the k best under (distance, index) are unique, and
+// a non-finite pose is never a candidate (it sets WK_DEV_NONFINITE).
 #include "wk_internal.cuh"
 
 namespace wk {
 namespace {
 
+constexpr int kScanMaxK = 64;
 constexpr int kScanThreads = 256;
 constexpr int kScanUnroll = 4;       // candidates per thread and round after the first
 constexpr int kScanLow = 256;        // a list longer than this is cut back to k at the end of the round
@@ -23,15 +36,24 @@ constexpr int kSelThreads = 512;     // scan_select: two blocks per SM, so that 
 constexpr int kScanWarm = 256;       // candidates of the first, list-seeding round
 constexpr int kPendLow = 256;        // survivors of the cheap bound are decided once this many have gathered
 constexpr int kScanCap = kScanLow + kSelThreads + 64;   // between two checks at most one entry per thread is added
-constexpr int kScanMaxK = 64;
 constexpr int kScanMaxBlocks = 1024;
-constexpr int kMergeThreads = 1024;
+
+constexpr int kSampleBlocks = 128;          // scan_sample's grid
+constexpr int kSampleThreads = 256;
+constexpr uint32_t kSurvivorCap = 1u << 20;  // entries of the survivor list
 
 struct ScanHeader {
   unsigned long long t_max_bits;     // max squared translation distance, as the bits of a non-negative double
   unsigned long long dot_min_bits;   // min |<q_cur, q_i>|, likewise
-  unsigned long long n_valid;
-  unsigned long long reserved;
+  uint32_t n_surv;                   // survivors appended so far (may exceed the capacity: then `overflow` is set)
+  uint32_t overflow;
+  uint32_t ticket;                   // blocks of the exact pass that have handed in their list
+  uint32_t pad;
+};
+// one record per scan_sample block
+struct SampleRecord {
+  double t_max;                              // largest squared translation distance among the block's samples
+  unsigned long long best[kScanMaxK];        // per class: (fp32 key bits << 32) | candidate index; ~0 = none
 };
 struct ScanEntry {
   double d;
@@ -58,38 +80,240 @@ __device__ __forceinline__ Cand candidate(const float4 a, const float4 b, const 
 
 struct Cur8 { float v[8]; };
 
-__global__ void scan_init(ScanHeader* h) {
-  dep_release();
-  h->t_max_bits = 0ull;
-  h->dot_min_bits = static_cast<unsigned long long>(__double_as_longlong(2.0));
-  h->n_valid = 0ull;
-  h->reserved = 0ull;
+// fp32 surrogates of a candidate's two terms, from the fp32 inputs: t32 = squared translation distance (relative error
+// below 1e-6), adot32 = |quaternion dot| (absolute error below 4e-7 for unit quaternions).
+__device__ __forceinline__ void cheap_terms(const float4 a, const float4 b, const float* cur, float& t32, float& adot32) {
+  const float dx = a.x - cur[0], dy = a.y - cur[1], dz = a.z - cur[2];
+  t32 = dx * dx + dy * dy + dz * dz;
+  adot32 = fabsf(b.x * cur[4] + b.y * cur[5] + b.z * cur[6] + b.w * cur[7]);
+}
+// lower bound of the rotation term 2 acos(|dot|): acos(x) >= sqrt(2 (1 - x)) on [0, 1]; 4e-7 covers the fp32 dot
+__device__ __forceinline__ float rot_lower_bound(float adot32) {
+  const float om = fmaxf(0.f, 1.f - adot32 - 4e-7f);
+  return 2.f * sqrtf(om + om) * (1.f - 3e-6f);
 }
 
-__global__ void __launch_bounds__(kScanThreads)
-scan_max(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, Cur8 cur, ScanHeader* h) {
+__global__ void __launch_bounds__(kSampleThreads)
+scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, int64_t n_samples, Cur8 cur,
+            int k, ScanHeader* __restrict__ h, SampleRecord* __restrict__ rec) {
+  __shared__ float s_tmax[kSampleThreads / 32];
+  __shared__ unsigned long long s_best[kScanMaxK];
+  dep_release();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (blockIdx.x == 0 && tid == 0) {   // the header fields scan_filter accumulates into
+    h->t_max_bits = 0ull;
+    h->dot_min_bits = static_cast<unsigned long long>(__double_as_longlong(2.0));
+    h->n_surv = 0u;
+    h->overflow = 0u;
+    h->ticket = 0u;
+  }
+  for (int g = tid; g < kScanMaxK; g += kSampleThreads) s_best[g] = ~0ull;
+  // sample s is candidate floor(s * n / n_samples) (integer arithmetic); block b takes samples b, b + gridDim.x, ...; class of a sample =
+  // its position in the block's sequence modulo k, so that classes are disjoint sets of candidates
+  const int64_t per_block = (n_samples + gridDim.x - 1) / gridDim.x;
+  // the weight pi / (largest t) of the key comes from the block's first 256 samples (any positive weight gives valid
+  // pivots, a rough one just picks slightly different ones); the record's t_max covers all of the block's samples
+  float tmax = 0.f;
+  {
+    const int64_t smp = static_cast<int64_t>(tid) * gridDim.x + blockIdx.x;
+    if (tid < per_block && smp < n_samples) {
+      const int64_t i = smp * n / n_samples;
+      if (!(valid && !__ldg(valid + i))) {
+        float t32, adot32;
+        cheap_terms(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v, t32, adot32);
+        if (t32 < 3.0e38f && adot32 < 3.0e38f) tmax = t32;   // false for NaN and Inf: not a candidate
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  if (lane == 0) s_tmax[warp] = tmax;
+  __syncthreads();
+  float est = s_tmax[0];
+  for (int w = 1; w < kSampleThreads / 32; ++w) est = fmaxf(est, s_tmax[w]);
+  __syncthreads();
+  const float wt = est > 0.f ? 3.14159274f / est : 0.f;
+  tmax = 0.f;
+  for (int64_t q = tid; q < per_block; q += kSampleThreads) {
+    const int64_t smp = q * gridDim.x + blockIdx.x;
+    if (smp >= n_samples) break;
+    const int64_t i = smp * n / n_samples;   // n_samples <= n: strictly increasing in smp, so samples are distinct
+    if (valid && !__ldg(valid + i)) continue;
+    float t32, adot32;
+    cheap_terms(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v, t32, adot32);
+    if (!(t32 < 3.0e38f && adot32 < 3.0e38f)) continue;
+    tmax = fmaxf(tmax, t32);
+    if (k > 0) {
+      const float om = fmaxf(0.f, 1.f - adot32);
+      const float key = 2.f * sqrtf(om + om) + wt * t32;   // ~ r + pi t / max t, non-negative
+      atomicMin(&s_best[static_cast<int>(q % k)],
+                (static_cast<unsigned long long>(__float_as_uint(key)) << 32) | static_cast<unsigned long long>(i));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+  if (lane == 0) s_tmax[warp] = tmax;
+  __syncthreads();
+  tmax = s_tmax[0];
+  for (int w = 1; w < kSampleThreads / 32; ++w) tmax = fmaxf(tmax, s_tmax[w]);
+  __syncthreads();
+  SampleRecord* my = rec + blockIdx.x;
+  if (tid == 0) my->t_max = static_cast<double>(tmax);
+  for (int g = tid; g < kScanMaxK; g += kSampleThreads) my->best[g] = s_best[g];
+}
+
+// The single pass over all poses.
+__global__ void __launch_bounds__(kScanThreads, 4)
+scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, Cur8 cur, int k,
+            const SampleRecord* __restrict__ rec, int n_rec, ScanHeader* __restrict__ h, uint32_t* __restrict__ surv,
+            uint32_t* __restrict__ status) {
+  __shared__ double s_t[kScanMaxK], s_r[kScanMaxK];
+  __shared__ float s_Tstar, s_Rstar, s_slope;
+  __shared__ double s_mt[kScanThreads / 32], s_md[kScanThreads / 32];
   dep_wait();
   dep_release();
-  double mt = 0.0, mdot = 2.0;
-  unsigned int cnt = 0;
-  for (int64_t i = static_cast<int64_t>(blockIdx.x) * kScanThreads + threadIdx.x; i < n;
-       i += static_cast<int64_t>(gridDim.x) * kScanThreads) {
-    if (valid && !__ldg(valid + i)) continue;
-    const Cand c = candidate(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v);
-    mt = fmax(mt, c.t);
-    mdot = fmin(mdot, c.adot);
-    ++cnt;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // ---- pivots: per class the best record over the sample blocks (four threads per class, a quarter of the records
+  // each), then the exact terms of those k candidates
+  __shared__ unsigned long long s_best[kScanMaxK];
+  if (tid < kScanMaxK) s_best[tid] = ~0ull;
+  __syncthreads();
+  {
+    const int g = tid & (kScanMaxK - 1), part = tid >> 6;   // 256 threads = 64 classes x 4 parts
+    if (g < k) {
+      unsigned long long best = ~0ull;
+      for (int b = part; b < n_rec; b += kScanThreads / kScanMaxK) {
+        const unsigned long long v = __ldcg(&rec[b].best[g]);
+        best = v < best ? v : best;
+      }
+      if (best != ~0ull) atomicMin(&s_best[g], best);
+    }
+    double tm = tid < n_rec ? __ldcg(&rec[tid].t_max) : 0.0;   // n_rec <= 128 < 256 threads
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) tm = fmax(tm, __shfl_xor_sync(0xffffffffu, tm, o));
+    if (lane == 0) s_mt[warp] = tm;
   }
+  __syncthreads();
+  if (tid < kScanMaxK) {
+    double t = -1.0, r = -1.0;   // negative: no pivot in this class
+    if (tid < k && s_best[tid] != ~0ull) {
+      const int64_t i = static_cast<int64_t>(s_best[tid] & 0xFFFFFFFFull);
+      const Cand c = candidate(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v);
+      if (isfinite(c.t) && isfinite(c.adot)) {
+        t = c.t;
+        r = 2.0 * acos(fmin(1.0, c.adot));
+      }
+    }
+    s_t[tid] = t;
+    s_r[tid] = r;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double mt_lo = 0.0;
+    for (int w = 0; w < kScanThreads / 32; ++w) mt_lo = fmax(mt_lo, s_mt[w]);
+    mt_lo *= 1.0 - 2e-6;   // the records hold fp32 values: below the true maximum after this
+    double Ts = 0.0, Rs = 0.0;
+    bool all = k > 0;
+    for (int g = 0; g < k; ++g) {
+      all = all && s_t[g] >= 0.0;
+      Ts = fmax(Ts, s_t[g]);
+      Rs = fmax(Rs, s_r[g]);
+    }
+    if (!all) {             // fewer than k pivots: nothing can be ruled out
+      s_Tstar = INFINITY;
+      s_Rstar = INFINITY;
+      s_slope = 0.f;
+    } else {                // every quantity rounded to the side that keeps more candidates
+      s_Tstar = Ts < 3.0e38 ? __double2float_ru(Ts * (1.0 + 1e-6)) : INFINITY;
+      s_Rstar = __double2float_ru(Rs * (1.0 + 1e-6));
+      s_slope = (Ts > 0.0 && mt_lo > 0.0) ? __double2float_ru(3.1415927 / mt_lo * (1.0 + 1e-6)) : (Ts > 0.0 ? INFINITY : 0.f);
+    }
+  }
+  __syncthreads();
+  const float Tstar = s_Tstar, Rstar = s_Rstar, slope = s_slope;
+  // ---- the stream
+  __shared__ uint32_t s_wbuf[kScanThreads / 32][64];
+  uint32_t* wbuf = s_wbuf[warp];
+  int wcnt = 0;                          // entries in the warp's buffer (the same value in all 32 lanes)
+  auto flush = [&]() {
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(&h->n_surv, static_cast<uint32_t>(wcnt));
+    base = __shfl_sync(0xffffffffu, base, 0);
+    for (int j = lane; j < wcnt; j += 32) {
+      if (base + j < kSurvivorCap) surv[base + j] = wbuf[j];
+      else h->overflow = 1u;
+    }
+    __syncwarp();
+  };
+  float rec_t = 0.f, rec_d = 2.f;        // this thread's fp32 records
+  double mt = 0.0, mdot = 2.0;           // exact maxima over the candidates whose fp32 value came near the record
+  bool bad = false;
+  const int64_t stride = static_cast<int64_t>(gridDim.x) * kScanThreads;
+  // the loop bound is the warp's first index, so that all 32 lanes make the same number of trips (the survivor
+  // bookkeeping below uses warp-wide votes); lanes past the end just have nothing live
+  for (int64_t i0 = static_cast<int64_t>(blockIdx.x) * kScanThreads + tid; i0 - lane < n; i0 += kScanUnroll * stride) {
+    float4 a[kScanUnroll], b[kScanUnroll];
+    bool live[kScanUnroll];
+#pragma unroll
+    for (int u = 0; u < kScanUnroll; ++u) {
+      const int64_t i = i0 + u * stride;
+      live[u] = i < n && !(valid && !__ldg(valid + i));
+      if (live[u]) {
+        a[u] = __ldg(poses + 2 * i);
+        b[u] = __ldg(poses + 2 * i + 1);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kScanUnroll; ++u) {
+      bool keep = false;
+      if (live[u]) {
+        float t32, adot32;
+        cheap_terms(a[u], b[u], cur.v, t32, adot32);
+        // exact terms only near a record (also for NaN / overflow, which fail both comparisons' negations)
+        if (!(t32 * (1.f + 4e-6f) < rec_t) || !(adot32 * (1.f - 4e-6f) - 2e-6f > rec_d)) {
+          const Cand c = candidate(a[u], b[u], cur.v);
+          if (isfinite(c.t) && isfinite(c.adot)) {
+            mt = fmax(mt, c.t);
+            mdot = fmin(mdot, c.adot);
+            rec_t = fmaxf(rec_t, t32);
+            rec_d = fminf(rec_d, adot32);
+          } else {
+            bad = true;
+            live[u] = false;
+          }
+        }
+        if (live[u]) {
+          const float gap = fmaxf(0.f, Tstar - t32 * (1.f - 3e-6f));
+          keep = !(rot_lower_bound(adot32) > Rstar + slope * gap);   // NaN on either side keeps the candidate
+        }
+      }
+      // survivors gather in a buffer of the warp's own (no block barrier anywhere in the stream); a full buffer takes
+      // consecutive places in the list with one atomic for the lot
+      const unsigned m = __ballot_sync(0xffffffffu, keep);
+      if (m) {
+        if (keep) wbuf[wcnt + __popc(m & ((1u << lane) - 1u))] = static_cast<uint32_t>(i0 + u * stride);
+        wcnt += __popc(m);
+        __syncwarp();
+        if (wcnt >= 32) {
+          flush();
+          wcnt = 0;
+        }
+      }
+    }
+  }
+  if (wcnt > 0) flush();
+  if (bad) atomicOr(status, WK_DEV_NONFINITE);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     mt = fmax(mt, __shfl_xor_sync(0xffffffffu, mt, o));
     mdot = fmin(mdot, __shfl_xor_sync(0xffffffffu, mdot, o));
-    cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
   }
-  if ((threadIdx.x & 31) == 0 && cnt > 0) {
+  if (lane == 0) { s_mt[warp] = mt; s_md[warp] = mdot; }
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kScanThreads / 32; ++w) { mt = fmax(mt, s_mt[w]); mdot = fmin(mdot, s_md[w]); }
     atomicMax(&h->t_max_bits, static_cast<unsigned long long>(__double_as_longlong(mt)));
     atomicMin(&h->dot_min_bits, static_cast<unsigned long long>(__double_as_longlong(mdot)));
-    atomicAdd(&h->n_valid, static_cast<unsigned long long>(cnt));
   }
 }
 
@@ -148,18 +372,27 @@ struct TopK {
 };
 
 __global__ void __launch_bounds__(kSelThreads, 2)
-scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, Cur8 cur,
-            const ScanHeader* __restrict__ h, int k, ScanEntry* __restrict__ block_out /*[gridDim.x][k]*/) {
+scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_all, int64_t n_all, Cur8 cur,
+            ScanHeader* __restrict__ h, const uint32_t* __restrict__ surv, int k,
+            ScanEntry* __restrict__ block_out /*[gridDim.x][k]*/, int out_capacity, int32_t* __restrict__ ids_out,
+            double* __restrict__ dist_out) {
   __shared__ unsigned long long s_key[2 * kScanCap];
   __shared__ int32_t s_i[2 * kScanCap];
-  __shared__ int32_t s_pend[kPendLow + kScanUnroll * kSelThreads];   // candidates that passed the cheap bound
+  __shared__ __align__(8) int32_t s_pend[kPendLow + kScanUnroll * kSelThreads];   // candidates that passed the cheap bound
   __shared__ int s_cnt, s_npend[2];
+  __shared__ uint32_t s_last;
+  __shared__ unsigned long long s_min;
   __shared__ double s_tau;
   __shared__ float s_tau_hi;
   dep_wait();
   dep_release();
   TopK top;
   top.init(s_key, s_i, &s_cnt, &s_tau, k);
+  // what is walked: the survivor list, or -- if it overflowed -- every pose (entry e is then candidate e)
+  const bool listed = h->overflow == 0u;
+  const int64_t n = listed ? static_cast<int64_t>(h->n_surv) : n_all;
+  const int32_t* valid = listed ? nullptr : valid_all;      // listed candidates have been checked already
+  auto cand_of = [&](int64_t e) -> int32_t { return listed ? static_cast<int32_t>(__ldg(surv + e)) : static_cast<int32_t>(e); };
   const double mt = __longlong_as_double(static_cast<long long>(h->t_max_bits));
   const double mr = 2.0 * acos(fmin(1.0, __longlong_as_double(static_cast<long long>(h->dot_min_bits))));
   // Cheap lower bound of the distance, in fp32 from the fp32 inputs: acos(x) >= sqrt(2 (1 - x)) on [0, 1], so
@@ -187,6 +420,7 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   // exact distance of one candidate, the arithmetic of retrieve_kernel
   auto exact = [&](int32_t i, double tau) {
     const Cand c = candidate(__ldg(poses + 2 * static_cast<int64_t>(i)), __ldg(poses + 2 * static_cast<int64_t>(i) + 1), cur.v);
+    if (!isfinite(c.t) || !isfinite(c.adot)) return;         // not a candidate (reported by the pass that read it first)
     const double rot = 2.0 * acos(fmin(1.0, c.adot));
     const double ta = mt > 0.0 ? c.t / mt : 0.0;
     const double rb = mr > 0.0 ? rot / mr : 0.0;
@@ -197,11 +431,16 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   refresh();
   // The first pass over kScanWarm candidates cuts the list at once: that gives a first k-th best, after which few of
   // the later candidates pass the bound.  Later rounds take kScanUnroll candidates per thread.
+  // (a survivor list needs no seeding: nearly all of it is wanted anyway, and the extra round trip to memory would
+  // only lengthen a short kernel)
   const int64_t warm0 = static_cast<int64_t>(blockIdx.x) * kScanWarm;
-  const int64_t warm_all = static_cast<int64_t>(gridDim.x) * kScanWarm;
-  if (k > 0 && threadIdx.x < kScanWarm) {
-    const int64_t i = warm0 + threadIdx.x;
-    if (i < n && !(valid && !__ldg(valid + i))) exact(static_cast<int32_t>(i), INFINITY);
+  const int64_t warm_all = listed ? 0 : static_cast<int64_t>(gridDim.x) * kScanWarm;
+  if (k > 0 && !listed && threadIdx.x < kScanWarm) {
+    const int64_t e = warm0 + threadIdx.x;
+    if (e < n) {
+      const int32_t i = cand_of(e);
+      if (!(valid && !__ldg(valid + i))) exact(i, INFINITY);
+    }
   }
   top.compact();
   refresh();
@@ -225,20 +464,27 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   };
   for (int64_t r = 0; r < rounds && k > 0; ++r) {
     float4 a[kScanUnroll], b[kScanUnroll];
+    int32_t ci[kScanUnroll];
     bool live[kScanUnroll];
 #pragma unroll
     for (int u = 0; u < kScanUnroll; ++u) {
-      const int64_t i = (r * kScanUnroll + u) * step + lane_off;
-      live[u] = i < n && !(valid && !__ldg(valid + i));
+      // a survivor list is dealt out entry by entry (block b takes entries b, b + gridDim.x, ...), so that a short list
+      // is shared by all blocks; a full scan takes whole 512-pose runs per block, for coalesced loads
+      const int64_t e = listed ? ((r * kScanUnroll + u) * kSelThreads + threadIdx.x) * gridDim.x + blockIdx.x
+                               : (r * kScanUnroll + u) * step + lane_off;
+      live[u] = e < n;
       if (live[u]) {
-        a[u] = __ldg(poses + 2 * i);
-        b[u] = __ldg(poses + 2 * i + 1);
+        ci[u] = cand_of(e);
+        live[u] = !(valid && !__ldg(valid + ci[u]));
+      }
+      if (live[u]) {
+        a[u] = __ldg(poses + 2 * static_cast<int64_t>(ci[u]));
+        b[u] = __ldg(poses + 2 * static_cast<int64_t>(ci[u]) + 1);
       }
     }
 #pragma unroll
     for (int u = 0; u < kScanUnroll; ++u)
-      if (live[u] && passes(a[u], b[u]))
-        s_pend[atomicAdd(&s_npend[0], 1)] = static_cast<int32_t>((r * kScanUnroll + u) * step + lane_off);
+      if (live[u] && passes(a[u], b[u])) s_pend[atomicAdd(&s_npend[0], 1)] = ci[u];
     // the thread whose push came last reads the final count, so the OR over the block cannot miss a full list
     if (__syncthreads_or(*reinterpret_cast<volatile int*>(&s_npend[0]) > kPendLow)) drain();
   }
@@ -250,99 +496,170 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
     o.d = e < s_cnt ? top.dist_at(e) : INFINITY;
     o.i = e < s_cnt ? s_i[e] : -1;
     o.pad = 0;
-    block_out[static_cast<int64_t>(blockIdx.x) * k + e] = o;
+    __stcg(reinterpret_cast<double2*>(block_out + static_cast<int64_t>(blockIdx.x) * k + e),
+           make_double2(o.d, __longlong_as_double((static_cast<long long>(static_cast<uint32_t>(o.pad)) << 32) |
+                                                  static_cast<uint32_t>(o.i))));
   }
-}
-
-// Merges the blocks' sorted lists: one thread per list holds its head; the block takes the smallest head k times.
-__global__ void __launch_bounds__(kMergeThreads)
-scan_merge(const ScanEntry* __restrict__ block_out, int n_lists, int k, int out_capacity, int32_t* __restrict__ ids_out,
-           double* __restrict__ dist_out) {
-  __shared__ unsigned long long s_wkey[kMergeThreads / 32];
-  __shared__ int32_t s_widx[kMergeThreads / 32];
-  __shared__ int s_wlist[kMergeThreads / 32];
-  __shared__ int s_winner;
-  dep_wait();
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // ---- hand in the list; the block that hands in last merges them all (nobody waits for anybody)
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&h->ticket, 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const int n_lists = static_cast<int>(gridDim.x);
+  const int tid = threadIdx.x;
   const unsigned long long kInf = static_cast<unsigned long long>(__double_as_longlong(INFINITY));
-  int pos = 0;   // head of this thread's list; the entry after it is fetched ahead, off the critical path
-  unsigned long long key, nkey;
-  int32_t idx, nidx;
-  auto load = [&](int at, unsigned long long& kk, int32_t& ii) {
-    kk = kInf;
-    ii = 0x7fffffff;
-    if (tid < n_lists && at < k) {
-      const ScanEntry x = block_out[static_cast<int64_t>(tid) * k + at];
-      if (x.i >= 0) { kk = static_cast<unsigned long long>(__double_as_longlong(x.d)); ii = x.i; }
-    }
+  auto entry = [&](int list, int e) -> ScanEntry {
+    const double2 v = __ldcg(reinterpret_cast<const double2*>(block_out + static_cast<int64_t>(list) * k + e));
+    ScanEntry x;
+    x.d = v.x;
+    x.i = static_cast<int32_t>(static_cast<uint32_t>(__double_as_longlong(v.y) & 0xFFFFFFFFll));
+    x.pad = 0;
+    return x;
   };
-  load(0, key, idx);
-  load(1, nkey, nidx);
-  for (int e = tid; e < out_capacity; e += kMergeThreads) {
+  for (int e = tid; e < out_capacity; e += blockDim.x) {
     ids_out[e] = -1;
     if (dist_out) dist_out[e] = 0.0;
   }
-  for (int out = 0; out < k; ++out) {
-    // smallest (distance, index) over the heads: warp shuffles, then the warps' winners
-    unsigned long long bk = key;
-    int32_t bi = idx;
-    int bl = tid;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk, o);
-      const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
-      if (ok < bk || (ok == bk && oi < bi)) { bk = ok; bi = oi; bl = ol; }
-    }
-    if (lane == 0) { s_wkey[warp] = bk; s_widx[warp] = bi; s_wlist[warp] = bl; }
-    __syncthreads();
-    if (warp == 0) {
-      bk = s_wkey[lane]; bi = s_widx[lane]; bl = s_wlist[lane];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const unsigned long long ok = __shfl_xor_sync(0xffffffffu, bk, o);
-        const int32_t oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        const int ol = __shfl_xor_sync(0xffffffffu, bl, o);
-        if (ok < bk || (ok == bk && oi < bi)) { bk = ok; bi = oi; bl = ol; }
+  if (tid == 0) { s_min = kInf; s_cnt = 0; h->ticket = 0u; }
+  __syncthreads();
+  if (k == 0) return;
+  // A list that holds k entries proves that k candidates lie within its last distance: nothing beyond the smallest such
+  // distance can be among the k best.  Every list is sorted, so what remains of it is a prefix.
+  // Likewise the k-th smallest of the lists' first entries: k candidates lie within it.  With candidates dealt to the
+  // blocks at random this is the sharper cut by far (it leaves little more than k entries).
+  unsigned long long* heads = reinterpret_cast<unsigned long long*>(s_pend);   // [n_lists] <= 1024 (s_pend is free by now)
+  for (int l = tid; l < n_lists; l += blockDim.x) {
+    const ScanEntry x = entry(l, k - 1);
+    if (x.i >= 0) atomicMin(&s_min, static_cast<unsigned long long>(__double_as_longlong(x.d)));
+    const ScanEntry f = entry(l, 0);
+    heads[l] = f.i >= 0 ? static_cast<unsigned long long>(__double_as_longlong(f.d)) : kInf;
+  }
+  __syncthreads();
+  if (n_lists >= k) {
+    for (int l = tid; l < n_lists; l += blockDim.x) {
+      const unsigned long long hl = heads[l];
+      int rank = 0;
+      for (int u = 0; u < n_lists; ++u) {
+        const unsigned long long hu = heads[u];
+        rank += (hu < hl) || (hu == hl && u < l);
       }
-      if (lane == 0) {
-        s_winner = (bi != 0x7fffffff) ? bl : -1;
-        if (bi != 0x7fffffff) {
-          ids_out[out] = bi;
-          if (dist_out) dist_out[out] = __longlong_as_double(static_cast<long long>(bk));
-        }
+      if (rank == k - 1 && hl != kInf) atomicMin(&s_min, hl);
+    }
+  }
+  __syncthreads();
+  const unsigned long long cut = s_min;
+  __syncthreads();   // heads (in s_pend) is dead from here on
+  constexpr int kGather = 2 * kScanCap;      // the two halves of the key / index arrays, free by now
+  for (int l = tid; l < n_lists; l += blockDim.x) {
+    for (int e = 0; e < k; ++e) {
+      const ScanEntry x = entry(l, e);
+      const unsigned long long key = static_cast<unsigned long long>(__double_as_longlong(x.d));
+      if (x.i < 0 || key > cut) break;
+      const int pos = atomicAdd(&s_cnt, 1);
+      if (pos < kGather) { s_key[pos] = key; s_i[pos] = x.i; }
+    }
+  }
+  __syncthreads();
+  const int n_g = s_cnt;
+  if (n_g <= kGather) {
+    // exact rank under (distance, index) among the gathered entries
+    for (int e = tid; e < n_g; e += blockDim.x) {
+      const unsigned long long ke = s_key[e];
+      const int32_t ie = s_i[e];
+      int rank = 0;
+      for (int u = 0; u < n_g; ++u) {
+        const unsigned long long ku = s_key[u];
+        rank += (ku < ke) || (ku == ke && s_i[u] < ie);
+      }
+      if (rank < k && rank < out_capacity) {
+        ids_out[rank] = ie;
+        if (dist_out) dist_out[rank] = __longlong_as_double(static_cast<long long>(ke));
+      }
+    }
+    return;
+  }
+  // Too many entries at or below the cut (many equal distances): take the smallest head of the lists k times.  Thread
+  // t walks lists t, t + blockDim.x, ...; s_pend holds each list's head position.
+  __shared__ int s_win_idx;
+  for (int l = tid; l < n_lists; l += blockDim.x) s_pend[l] = 0;
+  for (int out = 0; out < k && out < out_capacity; ++out) {
+    if (tid == 0) { s_min = kInf; s_win_idx = 0x7fffffff; }
+    __syncthreads();
+    for (int l = tid; l < n_lists; l += blockDim.x) {
+      if (s_pend[l] < k) {
+        const ScanEntry x = entry(l, s_pend[l]);
+        if (x.i >= 0) atomicMin(&s_min, static_cast<unsigned long long>(__double_as_longlong(x.d)));
       }
     }
     __syncthreads();
-    const int w = s_winner;
-    if (w < 0) break;          // every list is exhausted
-    if (tid == w) {
-      ++pos;
-      key = nkey;
-      idx = nidx;
-      load(pos + 1, nkey, nidx);
+    const unsigned long long best = s_min;
+    if (best == kInf) break;
+    for (int l = tid; l < n_lists; l += blockDim.x) {
+      if (s_pend[l] < k) {
+        const ScanEntry x = entry(l, s_pend[l]);
+        if (x.i >= 0 && static_cast<unsigned long long>(__double_as_longlong(x.d)) == best) atomicMin(&s_win_idx, x.i);
+      }
     }
+    __syncthreads();
+    const int win = s_win_idx;
+    for (int l = tid; l < n_lists; l += blockDim.x) {
+      if (s_pend[l] < k) {
+        const ScanEntry x = entry(l, s_pend[l]);
+        if (x.i == win) ++s_pend[l];
+      }
+    }
+    if (tid == 0) {
+      ids_out[out] = win;
+      if (dist_out) dist_out[out] = __longlong_as_double(static_cast<long long>(best));
+    }
+    __syncthreads();
   }
 }
 
 }  // namespace
 
-size_t retrieve_scan_scratch_bytes() {
-  return sizeof(ScanHeader) + static_cast<size_t>(kScanMaxBlocks) * kScanMaxK * sizeof(ScanEntry);
+namespace {
+struct ScanScratch {
+  ScanHeader* h;
+  SampleRecord* rec;
+  uint32_t* surv;
+  ScanEntry* block_out;
+  size_t total;
+};
+ScanScratch carve(void* base) {
+  ScanScratch sc;
+  uint8_t* p = static_cast<uint8_t*>(base);
+  size_t off = 0;
+  sc.h = reinterpret_cast<ScanHeader*>(p + off);        off += align_up(sizeof(ScanHeader), 256);
+  sc.rec = reinterpret_cast<SampleRecord*>(p + off);    off += align_up(sizeof(SampleRecord) * kSampleBlocks, 256);
+  sc.surv = reinterpret_cast<uint32_t*>(p + off);       off += align_up(sizeof(uint32_t) * kSurvivorCap, 256);
+  sc.block_out = reinterpret_cast<ScanEntry*>(p + off); off += static_cast<size_t>(kScanMaxBlocks) * kScanMaxK * sizeof(ScanEntry);
+  sc.total = off;
+  return sc;
 }
+}  // namespace
+
+size_t retrieve_scan_scratch_bytes() { return carve(nullptr).total; }
 
 wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* valid, int64_t n, const float* cur_pose,
                                int k, int32_t* ids_out, double* dist_out, int out_capacity, void* scratch, cudaStream_t s) {
-  ScanHeader* h = static_cast<ScanHeader*>(scratch);
-  ScanEntry* block_out = reinterpret_cast<ScanEntry*>(h + 1);
+  const ScanScratch sc = carve(scratch);
   Cur8 cur;
   for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose[i];
-  // pass 1: four resident 256-thread blocks per SM; pass 2: two resident 512-thread blocks per SM (fewer, longer lists
-  // to merge).  Fewer blocks when there is less than a round of work.
+  // the sample: one candidate in 64, at least 2^15 (all of them below that), at most 2^18
+  int64_t n_samples = n / 64;
+  if (n_samples < (1 << 15)) n_samples = (1 << 15);
+  if (n_samples > (1 << 18)) n_samples = (1 << 18);
+  if (n_samples > n) n_samples = n;
+  int sample_blocks = static_cast<int>((n_samples + kSampleThreads - 1) / kSampleThreads);
+  if (sample_blocks > kSampleBlocks) sample_blocks = kSampleBlocks;
+  if (sample_blocks < 1) sample_blocks = 1;
+  // the stream: four resident 256-thread blocks per SM; the exact pass: two resident 512-thread blocks per SM
   int64_t blocks = static_cast<int64_t>(ctx->sm_count) * 4;
   const int64_t needed = (n + kScanThreads - 1) / kScanThreads;
   if (blocks > needed) blocks = needed;
-  if (blocks > kScanMaxBlocks) blocks = kScanMaxBlocks;
   if (blocks < 1) blocks = 1;
   int64_t sel_blocks = static_cast<int64_t>(ctx->sm_count) * 2;
   const int64_t sel_needed = (n + kSelThreads - 1) / kSelThreads;
@@ -350,16 +667,14 @@ wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* v
   if (sel_blocks > kScanMaxBlocks) sel_blocks = kScanMaxBlocks;
   if (sel_blocks < 1) sel_blocks = 1;
   wk_status st;
-  scan_init<<<1, 1, 0, s>>>(h);
-  if ((st = after_launch(ctx)) != WK_OK) return st;
   const float4* p4 = reinterpret_cast<const float4*>(poses);
-  launch_chained(scan_max, dim3(static_cast<unsigned>(blocks)), dim3(kScanThreads), 0, s, p4, valid, n, cur, h);
+  scan_sample<<<sample_blocks, kSampleThreads, 0, s>>>(p4, valid, n, n_samples, cur, k, sc.h, sc.rec);
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  launch_chained(scan_select, dim3(static_cast<unsigned>(sel_blocks)), dim3(kSelThreads), 0, s, p4, valid, n, cur, h, k,
-                 block_out);
+  launch_chained(scan_filter, dim3(static_cast<unsigned>(blocks)), dim3(kScanThreads), 0, s, p4, valid, n, cur, k, sc.rec,
+                 sample_blocks, sc.h, sc.surv, ctx->status_dev);
   if ((st = after_launch(ctx)) != WK_OK) return st;
-  launch_chained(scan_merge, dim3(1), dim3(kMergeThreads), 0, s, block_out, static_cast<int>(sel_blocks), k, out_capacity,
-                 ids_out, dist_out);
+  launch_chained(scan_select, dim3(static_cast<unsigned>(sel_blocks)), dim3(kSelThreads), 0, s, p4, valid, n, cur, sc.h,
+                 sc.surv, k, sc.block_out, out_capacity, ids_out, dist_out);
   return after_launch(ctx);
 }
 

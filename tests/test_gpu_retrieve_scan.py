@@ -92,3 +92,59 @@ def test_scan_full_size(kv, log2n, k):
     n = 1 << log2n
     poses = wi.random_poses(100 + log2n, n + 1)
     _check(kv, poses[1:], poses[0], k)
+
+
+def test_scan_when_nothing_can_be_ruled_out(kv):
+    """Pure translation (every stored rotation equals the current one): no candidate can be ruled out before the
+    maxima are known, the survivor list overflows (more than 2^20 entries) and the call falls back to walking every pose
+    a second time.  The answer must not change."""
+    n = (1 << 20) + 300001
+    poses = wi.random_poses(55, n + 1)
+    poses[:, 4:8] = poses[0, 4:8]
+    _check(kv, poses[1:], poses[0], 16)
+    assert kv.poll_status() == (0, 0)
+
+
+def test_scan_on_a_camera_loop(kv):
+    """Poses along a jittered loop (neighbouring candidates are near-duplicates of each other), 300,000 of them."""
+    poses = wi.loop_poses(8, 300001)
+    _check(kv, poses[:-1].copy(), poses[-1], 8)
+    valid = wi.hash64(6, wi.STREAM_MISC, np.arange(300000)) % np.uint64(4) != 0
+    _check(kv, poses[:-1].copy(), poses[-1], 8, valid=valid)
+
+
+def test_scan_skips_non_finite_poses_and_reports_them(kv):
+    from paper_2605_22718_b200 import WK_DEV_NONFINITE, WK_ERR_NONFINITE
+    n = 70000
+    poses = wi.random_poses(77, n + 1)
+    P = poses[1:].copy()
+    bad = [5, 40000, 69999]
+    P[5, 0] = np.nan
+    P[40000, 6] = np.inf
+    P[69999, 2] = -np.inf
+    ok = np.ones(n, bool)
+    ok[bad] = False
+    Pd = torch.from_numpy(P).cuda()
+    ids = torch.empty(8, dtype=torch.int32, device="cuda")
+    dist = torch.empty(8, dtype=torch.float64, device="cuda")
+    kv.retrieve_scan(Pd, poses[0], 8, ids_out=ids, dist_out=dist)
+    st, flags = kv.poll_status()
+    assert st == WK_ERR_NONFINITE and flags & WK_DEV_NONFINITE
+    cand = np.nonzero(ok)[0]
+    ref_ids, ref_d, margin = o.retrieve(poses[0], P[cand], cand, 8)
+    assert margin > 1e-9
+    np.testing.assert_array_equal(ids.cpu().numpy(), ref_ids)
+    np.testing.assert_allclose(dist.cpu().numpy(), ref_d, rtol=0, atol=1e-12)
+
+
+def test_scan_many_equal_distances(kv):
+    """200,000 copies of one pose (all distances 0) and 200,000 copies of another: every block's list is full of ties,
+    far more entries tie at the cut than the merging block gathers at once, and the answer is still the lowest indices."""
+    poses = wi.random_poses(12, 3)
+    P = np.concatenate([np.repeat(poses[1][None], 200000, axis=0), np.repeat(poses[2][None], 200000, axis=0)])
+    got = _check(kv, P, poses[0], 16, need_margin=False)
+    d = o.retrieval_distances(poses[0], poses[1:3])
+    first = 0 if d[0] <= d[1] else 200000
+    assert got.tolist() == list(range(first, first + 16))
+    same = np.repeat(poses[0][None], 300000, axis=0)
+    assert _check(kv, same, poses[0], 64, need_margin=False).tolist() == list(range(64))
