@@ -182,21 +182,49 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return d;
 }
 // P = 2^(s * scale - m) for one row of a tile: rounds to bf16, stores into tensor memory over S (64 columns), returns
-// the fp32 row sum.  Every exponential goes to the MUFU: moving a share of them to a polynomial on the FMA pipe was
-// measured slower here (one softmax warp per SM sub-partition is latency-bound, not MUFU-throughput-bound).
+// the fp32 row sum.  The exponentials are the kernel's second bound (16 per clock and SM on the special-function unit,
+// as many clocks per tile as its tensor-core work), so kPoly of every 8 column pairs take 2^x from the FMA pipe instead:
+// x = n + f with n = round(x) by the add-a-large-constant trick, 2^f on [-1/2, 1/2] by a cubic (relative error 7.7e-5,
+// far inside the bf16 rounding P gets anyway: 2e-3), 2^n by adding n to the exponent field; all in packed fp32 pairs.
+// That path needs x >= -126 (it clamps at -120; such a weight is 1e-36 of the row's largest) and finite x, so tiles with
+// masked columns (-inf) take kPoly = 0.
 // kStore = false (LSE-only launches): only the row sum is wanted, nothing is written.
-template <bool kStore>
+#ifndef WK_ATTN_POLY
+#define WK_ATTN_POLY 2
+#endif
+template <bool kStore, int kPoly>
 __device__ __forceinline__ float exp_store_tile(const float (&s)[128], uint64_t scale2, uint64_t neg_m2, uint32_t tS) {
   uint64_t acc0 = 0, acc1 = 0, acc2 = 0, acc3 = 0;   // four independent (lo, hi) sums
+  const uint64_t magic2 = pack_f32x2(12582912.f, 12582912.f), nmagic2 = pack_f32x2(-12582912.f, -12582912.f);
+  const uint64_t mone2 = pack_f32x2(-1.f, -1.f);
+  const uint64_t c0 = pack_f32x2(0.9999289512634277f, 0.9999289512634277f);
+  const uint64_t c1 = pack_f32x2(0.6932762265205383f, 0.6932762265205383f);
+  const uint64_t c2 = pack_f32x2(0.242604061961174f, 0.242604061961174f);
+  const uint64_t c3 = pack_f32x2(0.055088773369789124f, 0.055088773369789124f);
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const uint64_t e = fma_f32x2(pack_f32x2(s[c * 32 + 2 * i], s[c * 32 + 2 * i + 1]), scale2, neg_m2);
-      float e0, e1;
+      float e0, e1, p0, p1;
       unpack_f32x2(e, e0, e1);
-      const float p0 = ex2_approx(e0), p1 = ex2_approx(e1);
+      if ((i & 7) < kPoly) {
+        const uint64_t x = pack_f32x2(fmaxf(e0, -120.f), fmaxf(e1, -120.f));
+        const uint64_t t = add_f32x2(x, magic2);                  // low mantissa bits = round(x)
+        const uint64_t f = fma_f32x2(add_f32x2(t, nmagic2), mone2, x);   // x - round(x), in [-1/2, 1/2]
+        uint64_t y = fma_f32x2(c3, f, c2);
+        y = fma_f32x2(y, f, c1);
+        y = fma_f32x2(y, f, c0);
+        float t0, t1, y0, y1;
+        unpack_f32x2(t, t0, t1);
+        unpack_f32x2(y, y0, y1);
+        p0 = __uint_as_float(__float_as_uint(y0) + (__float_as_uint(t0) << 23));
+        p1 = __uint_as_float(__float_as_uint(y1) + (__float_as_uint(t1) << 23));
+      } else {
+        p0 = ex2_approx(e0);
+        p1 = ex2_approx(e1);
+      }
       const uint64_t pp = pack_f32x2(p0, p1);
       if ((i & 3) == 0) acc0 = add_f32x2(acc0, pp);
       else if ((i & 3) == 1) acc1 = add_f32x2(acc1, pp);
@@ -571,7 +599,9 @@ memory_attention_kernel(const __grid_constant__ AttnParams p) {
           l *= alpha;
           const uint64_t neg_m2 = pack_f32x2(-m_used, -m_used);
           WK_PROF(3, blockIdx.x == 0 && tid == 0);
-          l += exp_store_tile<!kLse>(s, scale2, neg_m2, tS);   // masked columns hold -inf and come out as 0
+          // masked columns hold -inf and come out as 0 (special-function path only)
+          l += full_tile ? exp_store_tile<!kLse, WK_ATTN_POLY>(s, scale2, neg_m2, tS)
+                         : exp_store_tile<!kLse, 0>(s, scale2, neg_m2, tS);
           if (!kLse && __any_sync(0xffffffffu, rescale)) {
             // the previous P V product must have landed before O is touched
             if (!(ok = wait_or_abort(&bars.o_done[wg], (g - 1) & 1, &s_abort, p.status))) break;
