@@ -31,10 +31,19 @@ import wkinputs as wi  # noqa: E402
 METRIC = "memory-attn TFLOP/s over the whole chunk step (attention + retrieval + compression + pool append)"
 UNIT = "TFLOP/s"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per memory_attention_kernel launch from the ncu capture summarised in
-# profiles/memory_attention_cfg2_shape.md (cfg2 per-call shape: 122.7 MB read + 5.4 MB written); it does not depend on
-# the pool size, so the small-pool capture stands for the full workload.  Other workloads report null.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 128.1e6
+
+
+def ncu_traffic_bytes_per_launch(workload_name: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per memory_attention_kernel launch, from the figures file written
+    beside the ncu summary (profiles/memory_attention_cfg2_shape.json).  The capture ran on the cfg2 per-call shape with
+    a small pool; the traffic of a launch does not depend on the pool size, so it stands for every cfg2* workload.
+    Other workloads (and a missing file) report null."""
+    path = os.path.join(ROOT, "profiles", "memory_attention_cfg2_shape.json")
+    if not workload_name.startswith("cfg2") or not os.path.exists(path):
+        return None
+    with open(path) as f:
+        d = json.load(f)
+    return d["dram_bytes_read_per_launch"] + d["dram_bytes_write_per_launch"]
 
 
 def load_peaks():
@@ -126,7 +135,7 @@ class ChunkStepBench:
     """Holds the pool, the per-layer window buffers and rotating inputs of one workload, and runs chunk steps."""
 
     def __init__(self, w: wi.Workload, device_index: int, evict_sets: int = 4, e2e: bool = True, kv_splits: int = 0,
-                 prefill: bool = True):
+                 prefill: bool = True, max_splits: int = 8, max_k: int = 0):
         import torch
         from paper_2605_22718_b200 import WorldKV
         from wkinputs import device as wd
@@ -136,8 +145,8 @@ class ChunkStepBench:
         torch.cuda.set_device(self.dev)
         L, H, T, D = w.n_layers, w.n_heads, w.T, w.D
         self.kv = WorldKV(n_layers=L, n_heads=H, tokens_per_frame=T, n_keep=w.n_keep, pool_slots=w.pool_chunks,
-                          max_k=max(w.k, 1), max_dense_segments=1 + w.window_segments, device=device_index, max_batch=L, max_lq=w.Lq,
-                          max_splits=8)
+                          max_k=max(w.k, max_k, 1), max_dense_segments=1 + w.window_segments, device=device_index,
+                          max_batch=L, max_lq=w.Lq, max_splits=max_splits)
         bf = torch.bfloat16
         n_poses = w.pool_chunks + 4096
         if w.trajectory == "actions":
@@ -188,7 +197,7 @@ class ChunkStepBench:
             for s in range(S):
                 wd.query(self.Q[l, s], w.seed, l, s, 0)
         self.O = torch.empty_like(self.Q)
-        self.slots = torch.full((max(w.k, 1),), -1, dtype=torch.int32, device=self.dev)
+        self.slots = torch.full((max(w.k, max_k, 1),), -1, dtype=torch.int32, device=self.dev)
         self.step_no = 0
         self.attn_events = []
         self.e2e = e2e
@@ -239,12 +248,10 @@ class ChunkStepBench:
         if record_attention_events:
             e1.record()
             self.attn_events.append((e0, e1))
-        # the chunk leaving the window: compress every layer, evict the oldest stored chunk, append
+        # the chunk leaving the window: one call scores, selects, evicts the oldest stored chunk and stores the kept rows
         j = i % len(self.evK)
-        kv.compress_chunk(self.evK[j], keep_idx_out=self.keep)
-        if kv.pool_count() == w.pool_chunks:
-            kv.pool_evict(kv.pool_oldest())
-        kv.pool_append(0, w.n_layers, self.evK[j], self.evV[j], self.keep, pose, chunk_tag=w.pool_chunks + i)
+        kv.pool_compress_append(0, w.n_layers, self.evK[j], self.evV[j], pose, chunk_tag=w.pool_chunks + i,
+                                evict_oldest_if_full=True, keep_idx=self.keep)
 
     def time_steps(self, steps: int):
         """K chunk steps with every input already resident in HBM."""
@@ -260,15 +267,18 @@ class ChunkStepBench:
         barrier()
         return e0.elapsed_time(e1)
 
-    def isolated_attention(self):
+    def isolated_attention(self, k: int | None = None, kv_splits: int | None = None):
         """The attention call timed on its own, before the sustained steps heat the board into its power cap (the burst
-        peak it is set beside was measured the same way)."""
+        peak it is set beside was measured the same way).  k / kv_splits override the workload's retrieval budget and
+        the split setting (the sweeps of the LingBot-shaped and the full-history workloads)."""
         torch, w, kv = self.torch, self.w, self.kv
+        k = w.k if k is None else k
+        splits = self.kv_splits if kv_splits is None else kv_splits
         out = {}
         # the attention call timed on its own: 5 warm-up calls, then 24 timed ones whose Q / O / window rotate over the
         # layers' buffers (each call reads other memory than the one before it); median of per-call event times
         pose = self.poses[w.pool_chunks % len(self.poses)]
-        _, n_sl = kv.retrieve(pose, w.k, slots_out=self.slots)
+        _, n_sl = kv.retrieve(pose, k, slots_out=self.slots)
 
         def attn_call(i):
             l, s_ = i % w.n_layers, (i // w.n_layers) % w.denoise_steps
@@ -277,7 +287,7 @@ class ChunkStepBench:
                 rows = self.winK.shape[1] // w.window_segments
                 for q in range(w.window_segments):
                     segs.append((self.winK[l, q * rows:(q + 1) * rows], self.winV[l, q * rows:(q + 1) * rows]))
-            kv.memory_attention(l, self.Q[l, s_], segs, self.slots, n_sl, O=self.O[l, s_], kv_splits=self.kv_splits)
+            kv.memory_attention(l, self.Q[l, s_], segs, self.slots, n_sl, O=self.O[l, s_], kv_splits=splits)
 
         for i in range(5):
             attn_call(i)
@@ -288,7 +298,8 @@ class ChunkStepBench:
             b.record()
         torch.cuda.synchronize(self.dev)
         us = statistics.median(a.elapsed_time(b) for a, b in evs) * 1e3
-        out["attention_isolated"] = {"us_per_call": us, "tflops": self.attention_flops_per_call() / us / 1e6, "calls": 24}
+        out["attention_isolated"] = {"us_per_call": us, "tflops": w.attention_flops(k=min(k, n_sl)) / us / 1e6, "calls": 24,
+                                     "k": min(k, n_sl), "lkv": w.Lq + w.window_frames * w.T + min(k, n_sl) * w.C}
         return out["attention_isolated"]
 
     def side_metrics(self, iters: int = 20):
@@ -476,6 +487,74 @@ class OracleSample:
                 "est_step_ms": est_step_s * 1e3, "sample_seconds": t_attn + t_compress + t_retrieve}
 
 
+def oracle_attention_sample(w: wi.Workload, k: int, rows: int = 32):
+    """The oracle's attention on `rows` query rows of ONE head over the workload's KV length, inputs drawn for that
+    head's 128 columns only (seconds even at the LingBot width); scaled to all rows and heads.  Pool rows are the
+    leading C rows of generated chunks (the timing does not depend on which rows are kept)."""
+    from oracle import worldkv_oracle as o
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    cols = np.arange(128)
+    n_dense = w.Lq + w.window_frames * w.T
+    reps = (n_dense + w.F * w.T - 1) // (w.F * w.T)
+    Ks = [np.concatenate([wi.key_chunk_bf16(w.seed, 0, 100 + r, w.T, w.D, w.sigma, w.F, cols=cols) for r in range(reps)])[:n_dense]]
+    Vs = [np.concatenate([wi.value_chunk_bf16(w.seed, 0, 100 + r, w.T, w.D, w.F, cols=cols) for r in range(reps)])[:n_dense]]
+    for c in range(k):
+        Ks.append(wi.key_chunk_bf16(w.seed, 0, c, w.T, w.D, w.sigma, w.F, cols=cols)[:w.C])
+        Vs.append(wi.value_chunk_bf16(w.seed, 0, c, w.T, w.D, w.F, cols=cols)[:w.C])
+    K, V = np.concatenate(Ks)[:, None, :], np.concatenate(Vs)[:, None, :]
+    rows = min(rows, w.Lq)
+    Q = wi.query_bf16(w.seed, 0, 0, 0, w.Lq, w.D, cols=cols)[np.linspace(0, w.Lq - 1, rows).astype(np.int64)][:, None, :]
+    t0 = time.perf_counter()
+    o.attention(Q, K, V)
+    dt = time.perf_counter() - t0
+    est_call_s = dt * (w.Lq / rows) * w.n_heads
+    return {"value": 4.0 * w.Lq * K.shape[0] * 128 * w.n_heads / est_call_s / 1e12, "unit": UNIT, "cores": threads,
+            "kind": "oracle", "sample": f"{rows} of {w.Lq} query rows of one head over {K.shape[0]} KV tokens ({dt:.2f} s), "
+                                        f"scaled to all rows and {w.n_heads} heads"}
+
+
+def run_config_sweep(args):
+    """One JSON line per (workload, retrieval budget, KV split): the attention call timed on its own (median of 24
+    calls), for the single-layer benchmark workloads -- the Matrix-Game shape (cfg1), the LingBot shape at
+    k = 2, 4, 8, 16 (cfg3), the full one-minute history uncompressed and compressed at every split setting
+    (cfg4, cfg4c), and the paper's own window on both shapes."""
+    import torch
+    rank, local, world = dist_env()
+    if rank != 0:
+        return
+    peaks = load_peaks()
+    plan = [("cfg1", [None], [0]), ("cfg3", [2, 4, 8, 16], [0]), ("paper_mg", [None], [0]), ("paper_lb", [None], [0]),
+            ("cfg4", [None], [1, 2, 4, 8, 16, 0]), ("cfg4c", [None], [1, 2, 4, 8, 16, 0])]
+    only = set(args.sweep_only.split(",")) if args.sweep_only else None
+    for name, ks, splits_list in plan:
+        if only and name not in only:
+            continue
+        w = wi.WORKLOADS[name]
+        b = ChunkStepBench(w, local, e2e=False, max_splits=16, max_k=max([k or 0 for k in ks] + [w.k]))
+        sampler = ClockSampler(local)
+        for k in ks:
+            cpu = None if args.no_cpu_baseline else oracle_attention_sample(w, w.k if k is None else k)
+            for sp in splits_list:
+                sampler.start()
+                iso = b.isolated_attention(k=k, kv_splits=sp)
+                clocks = sampler.stop()
+                st, flags = b.kv.poll_status()
+                if st != 0:
+                    raise RuntimeError(f"device status {st} flags {flags}")
+                line = {"workload": name, "heads": w.n_heads, "tokens_per_frame": w.T, "lq": w.Lq, "k": iso["k"],
+                        "lkv": iso["lkv"], "kv_splits": sp, "us_per_call": iso["us_per_call"], "tflops": iso["tflops"],
+                        "frac_of_burst_peak": iso["tflops"] / peaks["bf16_tflops"],
+                        "frac_of_sustained_peak": iso["tflops"] / peaks["bf16_tflops_sustained"],
+                        "clocks": clocks, "cpu_baseline": cpu, "data": "synthetic"}
+                print(json.dumps(line), flush=True)
+        del b
+        torch.cuda.empty_cache()
+
+
 def run_reference(args, w: wi.Workload):
     rank, _, world = dist_env()
     if rank != 0:
@@ -491,7 +570,10 @@ def run_reference(args, w: wi.Workload):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": statistics.mean(t["est_step_ms"] for t in times),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "note": "CPU oracle on a bounded sample per step, scaled to one chunk step"},
+            "config": {"workload": w.name, "layers": w.n_layers, "denoise_steps": w.denoise_steps, "heads": w.n_heads,
+                       "tokens_per_frame": w.T, "lq": w.Lq, "lkv": w.Lkv, "pool_chunks": w.pool_chunks, "k": w.k,
+                       "l2": "inputs_larger_than_l2", "parallelism": "replicas" if world > 1 else "1gpu",
+                       "note": "CPU oracle on a bounded sample per step, scaled to one chunk step"},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": last["cores"], "kind": "oracle", "sample": last["sample"]},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0, "sample_seconds": statistics.mean(t["sample_seconds"] for t in times)}
@@ -540,6 +622,13 @@ def run_ours(args, w: wi.Workload):
     side = bench.side_metrics()
     side["compress"]["frac_of_hbm_peak"] = side["compress"]["gbs"] / peaks["hbm_gbs"]
     side["compress"]["peak_gbs"] = peaks["hbm_gbs"]
+    for key in ("2^16", "2^20", "2^24"):
+        side["retrieve_scan"][key]["frac_of_hbm_peak"] = side["retrieve_scan"][key]["gbs"] / peaks["hbm_gbs"]
+    lingbot = None
+    if w.name == "cfg2" and rank == 0 and not args.no_lingbot:
+        # the other model shape (1,560 tokens per frame, 40 heads): its attention call and its compression batch, timed
+        # on their own (a 3.8 GB pool beside the 61 GB one)
+        lingbot = lingbot_figures(local_rank, peaks)
     calls = bench.attention_calls_per_step()
     flops_call = bench.attention_flops_per_call()
     flops_step = flops_call * calls
@@ -549,7 +638,9 @@ def run_ours(args, w: wi.Workload):
         h2d = bench.hQ.numel() * 2 + bench.hcurK.numel() * 2 + bench.hcurV.numel() * 2
         d2h = bench.hO.numel() * 2
         e2e = {"value": world * flops_step / (ms_e2e / args.steps * 1e-3) / 1e12, "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps}
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps,
+               "note": "copied per step: Q and the denoising chunk's K/V in, O out; the window's K/V and the chunk "
+                       "leaving the window stay on the device, where a model produces them"}
     if rank != 0:
         return
     attn_launch_ms = statistics.mean(attn_ms) / calls
@@ -568,11 +659,13 @@ def run_ours(args, w: wi.Workload):
                       "tflops": achieved, "share_of_step": statistics.mean(attn_ms) / ms_per_step},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "frac_of_burst_peak": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " sustained",
-                     "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if w.name.startswith("cfg2") else None,
+                     "traffic": ncu_traffic_bytes_per_launch(w.name),
                      "kernel": "memory_attention_kernel"},
         "attention_isolated": dict(isolated, frac_of_burst_peak=isolated["tflops"] / peaks["bf16_tflops"]),
         "compress": side["compress"], "compress_per_head": side["compress_per_head"], "retrieve": side["retrieve"], "retrieve_query": side["retrieve_query"],
         "retrieve_scan": side["retrieve_scan"],
+        "attention_lingbot": None if lingbot is None else lingbot["attention"],
+        "compress_lingbot": None if lingbot is None else lingbot["compress"],
         "compress_append_bytes_per_step": comp_bytes,
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
     }
@@ -580,6 +673,47 @@ def run_ours(args, w: wi.Workload):
         cb = OracleSample(w).run(args.oracle_rows)
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
     print(json.dumps(line), flush=True)
+
+
+def lingbot_figures(device_index: int, peaks):
+    """cfg3 (LingBot-World-Fast shape, k = 8): the attention call timed on its own, and wk_compress_chunk over 40 layers'
+    worth of chunks (1.9 GB of keys per call)."""
+    import torch
+    from paper_2605_22718_b200 import WorldKV
+    from wkinputs import device as wd
+    w = wi.WORKLOADS["cfg3"]
+    b = ChunkStepBench(w, device_index, e2e=False)
+    iso = b.isolated_attention()
+    st, flags = b.kv.poll_status()
+    if st != 0:
+        raise RuntimeError(f"device status {st} flags {flags}")
+    out = {"attention": dict(iso, workload="cfg3", heads=w.n_heads, tokens_per_frame=w.T,
+                             frac_of_burst_peak=iso["tflops"] / peaks["bf16_tflops"])}
+    del b
+    torch.cuda.empty_cache()
+    batch = 40
+    kv = WorldKV(n_layers=1, n_heads=w.n_heads, tokens_per_frame=w.T, n_keep=w.n_keep, pool_slots=1, max_k=1,
+                 device=device_index, max_batch=batch)
+    sets = []
+    for i in range(3):
+        K = torch.empty((batch, w.F * w.T, w.D), dtype=torch.bfloat16, device=f"cuda:{device_index}")
+        for l in range(batch):
+            wd.key_chunk(K[l], w.seed, l, i, w.T, w.D, w.sigma, w.F)
+        sets.append(K)
+    keep = torch.empty((batch, w.C), dtype=torch.int32, device=f"cuda:{device_index}")
+    for i in range(3):
+        kv.compress_chunk(sets[i], keep_idx_out=keep)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(9):
+        kv.compress_chunk(sets[i % 3], keep_idx_out=keep)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / 9 * 1e3
+    nbytes = batch * w.F * w.T * w.D * 2
+    out["compress"] = {"us_per_call": us, "bytes_per_call": nbytes, "gbs": nbytes / us / 1e3, "problems": batch,
+                       "frac_of_hbm_peak": nbytes / us / 1e3 / peaks["hbm_gbs"], "workload": "cfg3 shape, 40 problems"}
+    return out
 
 
 def run_host_tier(args, w):
@@ -746,6 +880,18 @@ def run_retention_sweep(args, w):
                       "k": w.k, "data": "synthetic", "points": points}))
 
 
+def spawn_replicas(n: int) -> int:
+    """`bench.py --gpus N` started as a plain process: re-runs itself as N ranks (one per GPU) under torch.distributed.run
+    with the same arguments, so that N replicas are measured whichever way the script is started.  Returns the exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -760,13 +906,22 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--host-tier", action="store_true",
                     help="instead of the bench line: the chunk step with the stored chunks fetched from host memory")
+    ap.add_argument("--config-sweep", action="store_true",
+                    help="instead of the bench line: the attention call of cfg1, cfg3 (k sweep), cfg4 / cfg4c (split sweep) "
+                         "and the paper's window on both shapes, one JSON line each")
+    ap.add_argument("--sweep-only", default="", help="comma-separated workload names to restrict --config-sweep to")
+    ap.add_argument("--no-lingbot", action="store_true", help="skip the LingBot-shape figures of the default line")
     ap.add_argument("--retention-sweep", action="store_true",
                     help="instead of the bench line: chunk-step cost for n_keep in {0, T/4, T/2, T, 3T/2, 2T}")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))
     w = wi.WORKLOADS[args.workload]
-    if args.host_tier:
+    if args.config_sweep:
+        run_config_sweep(args)
+    elif args.host_tier:
         run_host_tier(args, w)
     elif args.retention_sweep:
         run_retention_sweep(args, w)

@@ -13,6 +13,7 @@
  *     D = n_heads * head_dim elements, base address 16-byte aligned.
  *   - Every call returns a wk_status: 0 on success, negative on error.  Errors that can be told from
  *     the arguments are returned before anything is launched and leave all state untouched.
+ *   - Every call that touches the device makes the context's device current (cudaSetDevice) first.
  *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*; NULL = legacy default
  *     stream) and is asynchronous.  Anomalies only the device can see (a stale slot id, a bounded
  *     wait that ran out, a non-finite score) set bits in a status word read with wk_poll_status.
@@ -120,6 +121,21 @@ wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_str
 wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
                          int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,
                          int64_t chunk_tag, int32_t* slot_io_host, void* stream);
+/* World Compression "applied once per chunk at storage time" (Section 4.3) as one call: for layers layer0 .. layer0+n-1
+ * scores the chunk's non-anchor keys (Eq. 5), selects the keep-sets and stores the kept rows of K and V in the pool --
+ * the same pool bytes, slot choice and bookkeeping as wk_compress_chunk followed by wk_pool_append, in one host call
+ * and one chain of launches: the gather is queued behind the selection on the device and walks the layers last to
+ * first, so that the keys the scoring pass touched last are gathered while L2 still holds them.
+ *   keep_idx_dev  [n][T + n_keep] int32 ([n][n_heads][T + n_keep] with WK_SCORE_PER_HEAD), caller-owned: receives the
+ *                 keep-sets (the gather reads them from there)
+ *   evict_oldest_if_full  non-zero: if this call has to pick a slot and none is free, the oldest stored chunk
+ *                 (wk_pool_oldest) is evicted first; *evicted_slot_host (may be NULL) receives its slot, else -1
+ *   slot_io_host, pose_host, chunk_tag  as in wk_pool_append (n <= max_batch; a chunk may be stored in several calls)
+ * Errors (all before anything is launched): WK_ERR_POOL_FULL, WK_ERR_BAD_SLOT, WK_ERR_SHAPE, WK_ERR_ARG, WK_ERR_UNBOUND. */
+wk_status wk_pool_compress_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
+                                  int64_t batch_stride_elems, int32_t* keep_idx_dev, const float* pose_host,
+                                  int64_t chunk_tag, int32_t evict_oldest_if_full, int32_t* slot_io_host,
+                                  int32_t* evicted_slot_host, void* stream);
 /* Frees a slot (stream-ordered: kernels already enqueued still see it).  WK_ERR_BAD_SLOT if not valid. */
 wk_status wk_pool_evict(wk_ctx* ctx, int32_t slot, void* stream);
 int32_t wk_pool_oldest(const wk_ctx* ctx);   /* valid slot with the earliest append, -1 if empty */
@@ -218,7 +234,8 @@ typedef struct {
  *   slots_dev [n_slots] int32 in device memory (e.g. wk_retrieve's output); an entry that is -1 is
  *             skipped silently, any other out-of-range or invalid entry is skipped and sets
  *             WK_DEV_BAD_SLOT; a slot listed twice is attended twice
- *   kv_splits 0 = cut the (head, 256-row query block) x KV-tile space into one equal range per SM (default);
+ *   kv_splits 0 = default: one CTA per (head, 256-row query block) when those fill at least three quarters of the SMs
+ *             (nothing is merged afterwards), else the (block x KV-tile) space cut into one equal range per SM;
  *             s in 1 .. max_splits = cut every block's KV range into s parts; -g = cut the whole space into g
  *             equal ranges (g CTAs; needs 2 g partial slots, see wk_scratch_bytes)
  * Errors: WK_ERR_SHAPE (lq > max_lq, n_slots > max_k, n_segs > max_dense_segments, kv_splits > max_splits),

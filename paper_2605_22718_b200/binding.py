@@ -63,6 +63,8 @@ def load_library() -> C.CDLL:
         "wk_bind": (i32, [vp, vp, sz, vp, sz, i32, i32, i32]),
         "wk_compress_chunk": (i32, [vp, vp, i64, i32, vp, vp, vp]),
         "wk_pool_append": (i32, [vp, i32, i32, vp, vp, i64, vp, C.POINTER(C.c_float), i64, C.POINTER(i32), vp]),
+        "wk_pool_compress_append": (i32, [vp, i32, i32, vp, vp, i64, vp, C.POINTER(C.c_float), i64, i32, C.POINTER(i32),
+                                          C.POINTER(i32), vp]),
         "wk_pool_evict": (i32, [vp, i32, vp]),
         "wk_pool_oldest": (i32, [vp]),
         "wk_pool_count": (i32, [vp]),
@@ -90,7 +92,7 @@ def load_library() -> C.CDLL:
 
 
 EXPORTED_SYMBOLS = ("wk_create", "wk_destroy", "wk_pool_bytes", "wk_scratch_bytes", "wk_bind", "wk_compress_chunk",
-                    "wk_pool_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
+                    "wk_pool_append", "wk_pool_compress_append", "wk_pool_evict", "wk_pool_oldest", "wk_pool_count", "wk_pool_tag", "wk_retrieve",
                     "wk_retrieve_noalloc", "wk_retrieve_query", "wk_retrieve_scan", "wk_retrieve_scan_scratch_bytes",
                     "wk_host_chunk_bytes", "wk_pool_store_host", "wk_pool_load_host",
                     "wk_memory_attention", "wk_poll_status", "wk_status_string", "wk_last_cuda_error",
@@ -196,6 +198,26 @@ class WorldKV:
         if st != WK_OK:
             raise WkError(st, "wk_pool_append")
         return slot_io.value
+
+    def pool_compress_append(self, layer0: int, n: int, K_chunks: torch.Tensor, V_chunks: torch.Tensor,
+                             pose: Sequence[float], chunk_tag: int = 0, slot: int = -1, evict_oldest_if_full: bool = False,
+                             keep_idx: Optional[torch.Tensor] = None, batch_stride_elems: Optional[int] = None,
+                             stream=None) -> Tuple[int, int, torch.Tensor]:
+        """wk_pool_compress_append: returns (slot, evicted slot or -1, keep_idx)."""
+        if batch_stride_elems is None:
+            batch_stride_elems = K_chunks.stride(0) if K_chunks.dim() == 3 else self.F * self.T * self.D
+        if keep_idx is None:
+            shape = (n, self.n_heads, self.C) if self.score_mode == SCORE_PER_HEAD else (n, self.C)
+            keep_idx = torch.empty(shape, dtype=torch.int32, device=self.device)
+        pose_arr = (C.c_float * 8)(*[float(x) for x in pose])
+        slot_io, evicted = C.c_int32(slot), C.c_int32(-1)
+        st = self.lib.wk_pool_compress_append(self.ctx, layer0, n, K_chunks.data_ptr(), V_chunks.data_ptr(),
+                                              batch_stride_elems, keep_idx.data_ptr(), pose_arr, chunk_tag,
+                                              1 if evict_oldest_if_full else 0, C.byref(slot_io), C.byref(evicted),
+                                              _stream(stream))
+        if st != WK_OK:
+            raise WkError(st, "wk_pool_compress_append")
+        return slot_io.value, evicted.value, keep_idx
 
     def pool_evict(self, slot: int, stream=None) -> None:
         st = self.lib.wk_pool_evict(self.ctx, slot, _stream(stream))

@@ -249,20 +249,15 @@ wk_status wk_compress_chunk(wk_ctx* ctx, const void* K_chunks, int64_t batch_str
                          scores_out, static_cast<cudaStream_t>(stream));
 }
 
-wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
-                         int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,
-                         int64_t chunk_tag, int32_t* slot_io_host, void* stream) {
-  if (!ctx || !K_chunks || !V_chunks || !keep_idx_dev || !pose_host || !slot_io_host) return WK_ERR_ARG;
-  if (!ctx->bound) return WK_ERR_UNBOUND;
-  WK_USE_DEVICE(ctx);
-  if (!aligned16(K_chunks) || !aligned16(V_chunks) || (batch_stride_elems & 7) != 0) return WK_ERR_ARG;
-  if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers) return WK_ERR_SHAPE;
-  if (n > 1 && batch_stride_elems < static_cast<int64_t>(ctx->FT) * ctx->D) return WK_ERR_ARG;
+// Shared by wk_pool_append and wk_pool_compress_append: slot choice and bookkeeping around the gather kernel.
+static wk_status append_checked(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
+                                int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,
+                                int64_t chunk_tag, int32_t* slot_io_host, cudaStream_t s, bool after_selection) {
   int slot = *slot_io_host;
   if (slot < 0) {
     if (slot != -1) return WK_ERR_BAD_SLOT;
-    for (int s = 0; s < ctx->cfg.pool_slots; ++s) {
-      if (ctx->slots[s].state == SLOT_FREE) { slot = s; break; }
+    for (int i = 0; i < ctx->cfg.pool_slots; ++i) {
+      if (ctx->slots[i].state == SLOT_FREE) { slot = i; break; }
     }
     if (slot < 0) return WK_ERR_POOL_FULL;
   } else {
@@ -272,9 +267,9 @@ wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_c
   for (int l = layer0; l < layer0 + n; ++l) {
     if (si.state == SLOT_OPEN && si.layer_mask[l]) return WK_ERR_BAD_SLOT;  // layer stored twice
   }
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
   wk_status st = launch_append(ctx, layer0, n, slot, static_cast<const __nv_bfloat16*>(K_chunks),
-                               static_cast<const __nv_bfloat16*>(V_chunks), batch_stride_elems, keep_idx_dev, s);
+                               static_cast<const __nv_bfloat16*>(V_chunks), batch_stride_elems, keep_idx_dev, s,
+                               after_selection);
   if (st != WK_OK) return st;
   if (si.state == SLOT_FREE) {
     si.state = SLOT_OPEN;
@@ -293,6 +288,56 @@ wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_c
   }
   *slot_io_host = slot;
   return WK_OK;
+}
+
+wk_status wk_pool_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
+                         int64_t batch_stride_elems, const int32_t* keep_idx_dev, const float* pose_host,
+                         int64_t chunk_tag, int32_t* slot_io_host, void* stream) {
+  if (!ctx || !K_chunks || !V_chunks || !keep_idx_dev || !pose_host || !slot_io_host) return WK_ERR_ARG;
+  if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
+  if (!aligned16(K_chunks) || !aligned16(V_chunks) || (batch_stride_elems & 7) != 0) return WK_ERR_ARG;
+  if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers) return WK_ERR_SHAPE;
+  if (n > 1 && batch_stride_elems < static_cast<int64_t>(ctx->FT) * ctx->D) return WK_ERR_ARG;
+  return append_checked(ctx, layer0, n, K_chunks, V_chunks, batch_stride_elems, keep_idx_dev, pose_host, chunk_tag,
+                        slot_io_host, static_cast<cudaStream_t>(stream), false);
+}
+
+wk_status wk_pool_compress_append(wk_ctx* ctx, int32_t layer0, int32_t n, const void* K_chunks, const void* V_chunks,
+                                  int64_t batch_stride_elems, int32_t* keep_idx_dev, const float* pose_host,
+                                  int64_t chunk_tag, int32_t evict_oldest_if_full, int32_t* slot_io_host,
+                                  int32_t* evicted_slot_host, void* stream) {
+  if (!ctx || !K_chunks || !V_chunks || !keep_idx_dev || !pose_host || !slot_io_host) return WK_ERR_ARG;
+  if (!ctx->bound) return WK_ERR_UNBOUND;
+  WK_USE_DEVICE(ctx);
+  if (!aligned16(K_chunks) || !aligned16(V_chunks) || (batch_stride_elems & 7) != 0) return WK_ERR_ARG;
+  if (layer0 < 0 || n < 1 || layer0 + n > ctx->cfg.n_layers || n > ctx->max_batch) return WK_ERR_SHAPE;
+  if (n > 1 && batch_stride_elems < static_cast<int64_t>(ctx->FT) * ctx->D) return WK_ERR_ARG;
+  if (evicted_slot_host) *evicted_slot_host = -1;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // everything that can fail on the host is settled before the first launch
+  int slot = *slot_io_host;
+  if (slot < -1 || slot >= ctx->cfg.pool_slots) return WK_ERR_BAD_SLOT;
+  if (slot >= 0) {
+    if (ctx->slots[slot].state != SLOT_OPEN) return WK_ERR_BAD_SLOT;
+    for (int l = layer0; l < layer0 + n; ++l)
+      if (ctx->slots[slot].layer_mask[l]) return WK_ERR_BAD_SLOT;
+  } else {
+    bool have_free = false;
+    for (const auto& si : ctx->slots) have_free = have_free || si.state == SLOT_FREE;
+    if (!have_free) {
+      const int victim = wk_pool_oldest(ctx);
+      if (!evict_oldest_if_full || victim < 0) return WK_ERR_POOL_FULL;
+      wk_status st = wk_pool_evict(ctx, victim, stream);
+      if (st != WK_OK) return st;
+      if (evicted_slot_host) *evicted_slot_host = victim;
+    }
+  }
+  wk_status st = launch_compress(ctx, static_cast<const __nv_bfloat16*>(K_chunks), batch_stride_elems, n, keep_idx_dev,
+                                 nullptr, s);
+  if (st != WK_OK) return st;
+  return append_checked(ctx, layer0, n, K_chunks, V_chunks, batch_stride_elems, keep_idx_dev, pose_host, chunk_tag,
+                        slot_io_host, s, true);
 }
 
 size_t wk_host_chunk_bytes(const wk_ctx* ctx) {

@@ -116,8 +116,10 @@ int attention_partial_slots(int n_heads, int max_lq, int max_splits);
 // Kernel launchers (one per translation unit).
 wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int batch, int32_t* keep_idx,
                           float* scores_out, cudaStream_t s);
+// after_selection: the launch is chained to the selection kernel that writes keep_idx (same stream, issued just before)
+// and walks the layers last to first.
 wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfloat16* K, const __nv_bfloat16* V,
-                        int64_t stride, const int32_t* keep_idx, cudaStream_t s);
+                        int64_t stride, const int32_t* keep_idx, cudaStream_t s, bool after_selection = false);
 wk_status launch_slot_mark(wk_ctx* ctx, int slot, int valid, const float* pose, cudaStream_t s);
 wk_status launch_retrieve(wk_ctx* ctx, const float* cur_pose, int k, int32_t* slots_out, double* dist_out, cudaStream_t s);
 // Kernels of one call that depend on each other in a chain are launched so that a kernel may be scheduled while its

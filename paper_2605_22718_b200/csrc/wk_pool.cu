@@ -12,8 +12,13 @@ constexpr int kAppendThreads = 256;
 __global__ void __launch_bounds__(kAppendThreads)
 append_rows(const __nv_bfloat16* __restrict__ Ksrc, const __nv_bfloat16* __restrict__ Vsrc, int64_t stride,
             const int32_t* __restrict__ keep_idx, int hs, int C, int FT, int D, __nv_bfloat16* __restrict__ Kdst,
-            __nv_bfloat16* __restrict__ Vdst, int64_t dst_layer_stride, int rows_per_cta, uint32_t* __restrict__ status) {
-  const int l = blockIdx.y, which = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+            __nv_bfloat16* __restrict__ Vdst, int64_t dst_layer_stride, int rows_per_cta, int reverse,
+            uint32_t* __restrict__ status) {
+  dep_wait();   // returns at once unless the launch was chained to the selection that writes keep_idx
+  // reverse: walk the layers last to first, so that the layers whose keys the scoring pass touched last (and L2 still
+  // holds) are gathered first
+  const int l = reverse ? static_cast<int>(gridDim.y) - 1 - static_cast<int>(blockIdx.y) : static_cast<int>(blockIdx.y);
+  const int which = blockIdx.z, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const __nv_bfloat16* src = (which ? Vsrc : Ksrc) + static_cast<int64_t>(l) * stride;
   __nv_bfloat16* dst = (which ? Vdst : Kdst) + static_cast<int64_t>(l) * dst_layer_stride;
   const int32_t* idx = keep_idx + static_cast<int64_t>(l) * hs * C;
@@ -42,7 +47,7 @@ __global__ void slot_mark(int32_t* __restrict__ valid, float* __restrict__ poses
 }  // namespace
 
 wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfloat16* K, const __nv_bfloat16* V,
-                        int64_t stride, const int32_t* keep_idx, cudaStream_t s) {
+                        int64_t stride, const int32_t* keep_idx, cudaStream_t s, bool after_selection) {
   const int C = ctx->C, D = ctx->D;
   const int64_t slot_elems = static_cast<int64_t>(C) * D;
   const int64_t layer_stride = slot_elems * ctx->cfg.pool_slots;
@@ -51,8 +56,12 @@ wk_status launch_append(wk_ctx* ctx, int layer0, int n, int slot, const __nv_bfl
   const int rows_per_cta = 32;
   const dim3 grid((C + rows_per_cta - 1) / rows_per_cta, n, 2);
   const int hs = ctx->cfg.score_mode == WK_SCORE_PER_HEAD ? ctx->cfg.n_heads : 1;
-  append_rows<<<grid, kAppendThreads, 0, s>>>(K, V, stride, keep_idx, hs, C, ctx->FT, D, Kdst, Vdst, layer_stride,
-                                              rows_per_cta, ctx->status_dev);
+  if (after_selection)
+    launch_chained(append_rows, grid, dim3(kAppendThreads), 0, s, K, V, stride, keep_idx, hs, C, ctx->FT, D, Kdst, Vdst,
+                   layer_stride, rows_per_cta, 1, ctx->status_dev);
+  else
+    append_rows<<<grid, kAppendThreads, 0, s>>>(K, V, stride, keep_idx, hs, C, ctx->FT, D, Kdst, Vdst, layer_stride,
+                                                rows_per_cta, 0, ctx->status_dev);
   return after_launch(ctx);
 }
 

@@ -8,7 +8,7 @@
 //       r_j > R* + (pi / mt_lo) * max(0, T* - t_j)
 // (a pivot with the larger translation term loses at most (T* - t_j) / mt_lo there and gains at least (r_j - R*) / pi).
 //
-//   scan_sample  a strided sample of the candidates (one in 64, 2^15 .. 2^18 of them): per block the largest t,
+//   scan_sample  a strided sample of the candidates (one in 128, 2^15 .. 2^18 of them): per block the largest t,
 //                and for each of k disjoint sample classes the candidate with the smallest r + pi t / (roughly max t),
 //                in fp32 -- pivots only have to be real candidates, not the best ones
 //   scan_filter  the single pass over all poses: every block first merges the sample blocks' records and takes the
@@ -52,7 +52,8 @@ struct ScanHeader {
 };
 // one record per scan_sample block
 struct SampleRecord {
-  double t_max;                              // largest squared translation distance among the block's samples
+  double t_max;                              // largest squared translation distance among the block's samples (fp32 value)
+  double dot_min;                            // smallest |quaternion dot| among them (fp32 value; 2 = none)
   unsigned long long best[kScanMaxK];        // per class: (fp32 key bits << 32) | candidate index; ~0 = none
 };
 struct ScanEntry {
@@ -96,7 +97,7 @@ __device__ __forceinline__ float rot_lower_bound(float adot32) {
 __global__ void __launch_bounds__(kSampleThreads)
 scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid, int64_t n, int64_t n_samples, Cur8 cur,
             int k, ScanHeader* __restrict__ h, SampleRecord* __restrict__ rec) {
-  __shared__ float s_tmax[kSampleThreads / 32];
+  __shared__ float s_tmax[kSampleThreads / 32], s_dmin[kSampleThreads / 32];
   __shared__ unsigned long long s_best[kScanMaxK];
   dep_release();
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -134,6 +135,7 @@ scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   __syncthreads();
   const float wt = est > 0.f ? 3.14159274f / est : 0.f;
   tmax = 0.f;
+  float dmin = 2.f;
   for (int64_t q = tid; q < per_block; q += kSampleThreads) {
     const int64_t smp = q * gridDim.x + blockIdx.x;
     if (smp >= n_samples) break;
@@ -143,6 +145,7 @@ scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
     cheap_terms(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v, t32, adot32);
     if (!(t32 < 3.0e38f && adot32 < 3.0e38f)) continue;
     tmax = fmaxf(tmax, t32);
+    dmin = fminf(dmin, adot32);
     if (k > 0) {
       const float om = fmaxf(0.f, 1.f - adot32);
       const float key = 2.f * sqrtf(om + om) + wt * t32;   // ~ r + pi t / max t, non-negative
@@ -151,14 +154,18 @@ scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
     }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-  if (lane == 0) s_tmax[warp] = tmax;
+  for (int o = 16; o > 0; o >>= 1) {
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    dmin = fminf(dmin, __shfl_xor_sync(0xffffffffu, dmin, o));
+  }
+  if (lane == 0) { s_tmax[warp] = tmax; s_dmin[warp] = dmin; }
   __syncthreads();
   tmax = s_tmax[0];
-  for (int w = 1; w < kSampleThreads / 32; ++w) tmax = fmaxf(tmax, s_tmax[w]);
+  dmin = s_dmin[0];
+  for (int w = 1; w < kSampleThreads / 32; ++w) { tmax = fmaxf(tmax, s_tmax[w]); dmin = fminf(dmin, s_dmin[w]); }
   __syncthreads();
   SampleRecord* my = rec + blockIdx.x;
-  if (tid == 0) my->t_max = static_cast<double>(tmax);
+  if (tid == 0) { my->t_max = static_cast<double>(tmax); my->dot_min = static_cast<double>(dmin); }
   for (int g = tid; g < kScanMaxK; g += kSampleThreads) my->best[g] = s_best[g];
 }
 
@@ -168,7 +175,7 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
             const SampleRecord* __restrict__ rec, int n_rec, ScanHeader* __restrict__ h, uint32_t* __restrict__ surv,
             uint32_t* __restrict__ status) {
   __shared__ double s_t[kScanMaxK], s_r[kScanMaxK];
-  __shared__ float s_Tstar, s_Rstar, s_slope;
+  __shared__ float s_Tstar, s_Rstar, s_slope, s_rec_t, s_rec_d;
   __shared__ double s_mt[kScanThreads / 32], s_md[kScanThreads / 32];
   dep_wait();
   dep_release();
@@ -189,9 +196,13 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
       if (best != ~0ull) atomicMin(&s_best[g], best);
     }
     double tm = tid < n_rec ? __ldcg(&rec[tid].t_max) : 0.0;   // n_rec <= 128 < 256 threads
+    double dm = tid < n_rec ? __ldcg(&rec[tid].dot_min) : 2.0;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) tm = fmax(tm, __shfl_xor_sync(0xffffffffu, tm, o));
-    if (lane == 0) s_mt[warp] = tm;
+    for (int o = 16; o > 0; o >>= 1) {
+      tm = fmax(tm, __shfl_xor_sync(0xffffffffu, tm, o));
+      dm = fmin(dm, __shfl_xor_sync(0xffffffffu, dm, o));
+    }
+    if (lane == 0) { s_mt[warp] = tm; s_md[warp] = dm; }
   }
   __syncthreads();
   if (tid < kScanMaxK) {
@@ -209,8 +220,11 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   }
   __syncthreads();
   if (tid == 0) {
-    double mt_lo = 0.0;
-    for (int w = 0; w < kScanThreads / 32; ++w) mt_lo = fmax(mt_lo, s_mt[w]);
+    double mt_lo = 0.0, md_hi = 2.0;
+    for (int w = 0; w < kScanThreads / 32; ++w) { mt_lo = fmax(mt_lo, s_mt[w]); md_hi = fmin(md_hi, s_md[w]); }
+    // the sample's records seed every thread's: a candidate below them (by more than fp32 rounding) cannot hold a maximum
+    s_rec_t = static_cast<float>(mt_lo);
+    s_rec_d = static_cast<float>(md_hi);
     mt_lo *= 1.0 - 2e-6;   // the records hold fp32 values: below the true maximum after this
     double Ts = 0.0, Rs = 0.0;
     bool all = k > 0;
@@ -245,7 +259,7 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
     }
     __syncwarp();
   };
-  float rec_t = 0.f, rec_d = 2.f;        // this thread's fp32 records
+  float rec_t = s_rec_t, rec_d = s_rec_d;   // this thread's fp32 records, seeded with the sample's
   double mt = 0.0, mdot = 2.0;           // exact maxima over the candidates whose fp32 value came near the record
   bool bad = false;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * kScanThreads;
@@ -648,8 +662,8 @@ wk_status launch_retrieve_scan(wk_ctx* ctx, const float* poses, const int32_t* v
   const ScanScratch sc = carve(scratch);
   Cur8 cur;
   for (int i = 0; i < 8; ++i) cur.v[i] = cur_pose[i];
-  // the sample: one candidate in 64, at least 2^15 (all of them below that), at most 2^18
-  int64_t n_samples = n / 64;
+  // the sample: one candidate in 128, at least 2^15 (all of them below that), at most 2^18
+  int64_t n_samples = n / 128;
   if (n_samples < (1 << 15)) n_samples = (1 << 15);
   if (n_samples > (1 << 18)) n_samples = (1 << 18);
   if (n_samples > n) n_samples = n;

@@ -43,3 +43,17 @@ def test_reference_arm_prints_one_json_line_on_rank_0_only():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     out = subprocess.run(cmd, capture_output=True, text=True, check=True, env=env).stdout.strip()
     assert out == ""
+
+
+def test_gpus_flag_without_torchrun_spawns_the_ranks_itself():
+    """`bench.py --gpus 2` started as a plain process re-runs itself as two ranks; rank 0's line says n_gpus = 2 and the
+    other rank prints nothing (the reference arm needs no GPU, so this runs on CPU)."""
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "cfg0", "--steps", "1",
+           "--warmup", "0", "--gpus", "2"]
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    res = subprocess.run(cmd, capture_output=True, text=True, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.strip().splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["config"]["parallelism"] == "replicas"

@@ -245,3 +245,56 @@ def test_argument_errors_are_reported_before_launch():
         kv.compress_chunk(torch.zeros((2, 48, 128), dtype=torch.bfloat16, device="cuda"))
     assert e.value.status == WK_ERR_SHAPE
     assert kv.launch_count() == n0
+
+
+@pytest.mark.parametrize("per_head", [False, True])
+def test_compress_append_in_one_call_stores_the_same_pool_bytes(per_head):
+    """wk_pool_compress_append against wk_compress_chunk + wk_pool_append (same slots, same stored rows, same keep-sets)
+    and against the oracle's pool model, including the evict-oldest-when-full path and a chunk stored in two calls."""
+    from paper_2605_22718_b200 import WkError, WK_ERR_POOL_FULL, SCORE_PER_HEAD
+    T, H, n_keep, L, slots = 40, 3, 21, 4, 3
+    D, C_rows = H * 128, T + n_keep
+    mode = SCORE_PER_HEAD if per_head else 0
+    kw = dict(n_layers=L, n_heads=H, tokens_per_frame=T, n_keep=n_keep, pool_slots=slots, max_k=slots, max_batch=L,
+              score_mode=mode)
+    kv_a, kv_b = make_kv(**kw), make_kv(**kw)
+    ref = Scenario(kv_b, 13, 0.1, L, T, H, n_keep, slots, per_head=per_head)
+    poses = wi.random_poses(13, 6)
+    pool_words = 2 * L * slots * C_rows * D            # K then V, bf16 elements
+
+    def store_fused(chunk, **extra):
+        K, V = ref.chunk_bits(chunk)
+        Kd, Vd = wd.to_device_bf16(np.stack(K)), wd.to_device_bf16(np.stack(V))
+        return kv_a.pool_compress_append(0, L, Kd, Vd, poses[chunk], chunk_tag=chunk, **extra)
+
+    for c in range(3):
+        slot, evicted, keep = store_fused(c)
+        assert ref.append_chunk(c, poses[c]) == slot and evicted == -1     # Scenario checks kv_b's keep-sets vs the oracle
+        ref_keep = [o.compress_chunk_per_head(k, T, n_keep, H)[0] if per_head else o.compress_chunk(k, T, n_keep)[0]
+                    for k in ref.chunk_bits(c)[0]]
+        np.testing.assert_array_equal(keep.cpu().numpy(), np.stack(ref_keep))
+    a = kv_a.pool[:pool_words * 2].view(torch.int16)
+    b = kv_b.pool[:pool_words * 2].view(torch.int16)
+    assert torch.equal(a, b)
+    # full pool: refused without the flag (and nothing launched), oldest evicted with it
+    n0 = kv_a.launch_count()
+    with pytest.raises(WkError) as e:
+        store_fused(3)
+    assert e.value.status == WK_ERR_POOL_FULL and kv_a.launch_count() == n0
+    slot, evicted, _ = store_fused(3, evict_oldest_if_full=True)
+    assert (slot, evicted) == (0, 0) and kv_a.pool_tag(0) == 3 and kv_a.pool_count() == 3
+    kv_b.pool_evict(0); ref.pool.evict(0)
+    assert ref.append_chunk(3, poses[3]) == 0
+    assert torch.equal(kv_a.pool[:pool_words * 2].view(torch.int16), kv_b.pool[:pool_words * 2].view(torch.int16))
+    # a chunk stored in two calls (layers 0-1, then 2-3) becomes visible after the second
+    kv_a.pool_evict(1)
+    K, V = ref.chunk_bits(4)
+    Kd, Vd = wd.to_device_bf16(np.stack(K)), wd.to_device_bf16(np.stack(V))
+    slot, _, _ = kv_a.pool_compress_append(0, 2, Kd[:2], Vd[:2], poses[4], chunk_tag=4)
+    assert slot == 1 and kv_a.pool_count() == 2
+    slot2, _, _ = kv_a.pool_compress_append(2, 2, Kd[2:], Vd[2:], poses[4], chunk_tag=4, slot=slot)
+    assert slot2 == 1 and kv_a.pool_count() == 3 and kv_a.pool_tag(1) == 4
+    kv_b.pool_evict(1); ref.pool.evict(1)
+    assert ref.append_chunk(4, poses[4]) == 1
+    assert torch.equal(kv_a.pool[:pool_words * 2].view(torch.int16), kv_b.pool[:pool_words * 2].view(torch.int16))
+    assert kv_a.poll_status() == (0, 0) and kv_b.poll_status() == (0, 0)
