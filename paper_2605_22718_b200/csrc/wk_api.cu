@@ -38,7 +38,7 @@ ScratchLayout scratch_layout(const wk_config& c, int max_batch, int max_lq, int 
   s.mnorm_off = off; off += align_up(B * 32 * sizeof(double), 256);   // up to 32 shares of |m|^2 per problem
   s.part_off = off;  off += align_up(Bc * s.anchor_parts * D * sizeof(double), 256);
   s.inv_off = off;   off += align_up(B * c.tokens_per_frame * sizeof(double), 256);
-  s.cnt_off = off;   off += align_up(2 * Bc * sizeof(uint32_t), 256);   // tickets of the anchor and the score pass
+  s.cnt_off = off;   off += align_up((3 * Bc + 4) * sizeof(uint32_t), 256);   // tickets of the anchor and the score pass, ready words, work queue
   s.dist_off = off;  off += align_up(static_cast<size_t>(c.pool_slots) * 2 * sizeof(double), 256);
   const size_t slots = static_cast<size_t>(attention_partial_slots(c.n_heads, max_lq > 0 ? max_lq : 1, max_splits));
   s.opart_off = off;   off += align_up(slots * 2 * kTileQ * kHeadDim * sizeof(float), 256);

@@ -203,17 +203,19 @@ __device__ __forceinline__ void group_accumulate(const uint8_t* buf, size_t row_
   }
 }
 
+// The work of one anchor CTA (slice `part` of `parts` of chunk b).  `ready` (may be null): a word per chunk that the last
+// CTA of the chunk sets to `epoch` once m64 / m32 / |m|^2 are written, for score CTAs of the same launch to poll.
 template <int VPT>
-__global__ void __launch_bounds__(kAnchorThreads, VPT == 1 ? 4 : (VPT == 2 ? 3 : 2))
-anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int hs, int G, int rpp,
-            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
-            float* __restrict__ m32, double* __restrict__ mnorm2, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bar[2];
+__device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int parts, const __nv_bfloat16* __restrict__ K,
+                                            int64_t stride, int T, int D, int hs, int G, int rpp,
+                                            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets,
+                                            double* __restrict__ m64, float* __restrict__ m32, double* __restrict__ mnorm2,
+                                            uint32_t* __restrict__ status, uint32_t* ready, uint32_t epoch,
+                                            uint64_t* bar, uint32_t& gbase) {
+  // bar[2]: the caller's two mbarriers (initialised once per CTA, count 1); gbase: bulk copies this CTA has waited for so
+  // far -- copy number n lands in buffer n & 1 and completes phase n >> 1 of barrier n & 1
   __shared__ uint32_t s_flag;
   __shared__ double red[kAnchorWarps];
-  dep_release();
-  const int b = blockIdx.y, part = blockIdx.x, parts = gridDim.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const size_t row_bytes = static_cast<size_t>(D) * 2;
   const int nseg = kAnchorWarps / G;                                        // column segments per row in phase 1
@@ -224,19 +226,17 @@ anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, i
   const int r0 = min(T, part * rpp), r1 = min(T, r0 + rpp);
   const int n_groups = (r1 - r0 + G - 1) / G;
   const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride;
-  if (tid == 0) {
-    ptx::mbar_init(&bar[0], 1);
-    ptx::mbar_init(&bar[1], 1);
-    ptx::fence_mbar_init();
-  }
-  __syncthreads();
   auto issue = [&](int g) {   // thread 0: one bulk copy of the group's rows (contiguous in memory)
     const int ra = r0 + g * G;
     const uint32_t bytes = static_cast<uint32_t>(min(G, r1 - ra) * row_bytes);
-    ptx::mbar_expect_tx(&bar[g & 1], bytes);
-    ptx::bulk_load_1d(rows_s + (g & 1) * G * row_bytes, Kb + static_cast<int64_t>(ra) * D, bytes, &bar[g & 1]);
+    const uint32_t n = gbase + g;
+    ptx::mbar_expect_tx(&bar[n & 1], bytes);
+    ptx::bulk_load_1d(rows_s + (n & 1) * G * row_bytes, Kb + static_cast<int64_t>(ra) * D, bytes, &bar[n & 1]);
   };
-  if (tid == 0 && n_groups > 0) issue(0);
+  if (tid == 0 && n_groups > 0) {
+    ptx::fence_proxy_async_smem();   // the buffers may have been written with ordinary stores by the work item before
+    issue(0);
+  }
   double acc[8 * VPT];
 #pragma unroll
   for (int i = 0; i < 8 * VPT; ++i) acc[i] = 0.0;
@@ -249,17 +249,28 @@ anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, i
       if (tid == 0) issue(g + 1);     // its buffer was released by the barrier that ended group g - 1
       armed = g + 2;
     }
-    const bool landed = ptx::mbar_wait(&bar[g & 1], (g >> 1) & 1);
+    const uint32_t n_cur = gbase + g;
+    const bool landed = ptx::mbar_wait(&bar[n_cur & 1], (n_cur >> 1) & 1);
     if (__syncthreads_or(!landed)) {  // a copy that never lands: report, stop reading, still hand in the slice
       if (tid == 0) atomicOr(status, WK_DEV_TIMEOUT);
       break;
     }
     const int rows = min(G, r1 - (r0 + g * G));
-    const uint8_t* buf = rows_s + (g & 1) * G * row_bytes;
+    const uint8_t* buf = rows_s + (n_cur & 1) * G * row_bytes;
     // ---- phase 1: norms (integer-pipe conversions; redone exactly when a norm falls outside the safe range)
     group_norms<false>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
-    __syncthreads();
     bool redo = false;
+    if (hs == 1 && nseg == 1) {
+      // one warp holds a whole row's squared norm: its first lane finishes the row on the spot, so that the eight
+      // reciprocal square roots run side by side and one barrier (the vote below) ends the phase
+      if (warp < rows && lane == 0) {
+        const double n2 = n2_s[warp * n2_pitch];
+        inv_s[warp] = n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);
+        redo = !(n2 >= kNorm2Lo && n2 <= kNorm2Hi);
+      }
+    } else {
+      __syncthreads();
+    }
     auto finish_norms = [&](bool check) {
       for (int i = tid; i < rows * hs; i += kAnchorThreads) {
         const int r = i / hs, h = i - r * hs;
@@ -270,7 +281,7 @@ anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, i
         if (check) redo = redo || !(n2 >= kNorm2Lo && n2 <= kNorm2Hi);
       }
     };
-    finish_norms(true);
+    if (!(hs == 1 && nseg == 1)) finish_norms(true);
     const bool exact = __syncthreads_or(redo) != 0;
     if (exact) {
       group_norms<true>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
@@ -288,8 +299,10 @@ anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, i
   if (tid == 0) {
     for (int gg = g; gg < armed; ++gg)   // empty unless the loop was left at group g < n_groups
       for (uint32_t i = 0; i < (1u << 16); ++i)
-        if (ptx::mbar_try_wait(&bar[gg & 1], (gg >> 1) & 1)) break;
+        if (ptx::mbar_try_wait(&bar[(gbase + gg) & 1], ((gbase + gg) >> 1) & 1)) break;
   }
+  gbase += static_cast<uint32_t>(armed);   // every issued copy has been waited for (or given up on) by now
+  __syncthreads();
   // ---- this CTA's slice
   double* my = partial + (static_cast<int64_t>(b) * max_parts + part) * D;
 #pragma unroll
@@ -359,7 +372,34 @@ anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, i
       mnorm2[static_cast<int64_t>(b) * kMaxNormParts] = t;
     }
   }
-  if (tid == 0) tickets[b] = 0;   // ready for the next call
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    tickets[b] = 0;   // ready for the next call
+    if (ready) {
+      __threadfence();                                   // m64 / m32 / |m|^2 of every thread are out before the flag
+      *reinterpret_cast<volatile uint32_t*>(ready + b) = epoch;
+    }
+  }
+}
+
+template <int VPT>
+__global__ void __launch_bounds__(kAnchorThreads, VPT == 1 ? 4 : (VPT == 2 ? 3 : 2))
+anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int hs, int G, int rpp,
+            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
+            float* __restrict__ m32, double* __restrict__ mnorm2, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bar[2];
+  dep_release();
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bar[0], 1);
+    ptx::mbar_init(&bar[1], 1);
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  uint32_t gbase = 0;
+  anchor_role<VPT>(smem, blockIdx.y, blockIdx.x, gridDim.x, K, stride, T, D, hs, G, rpp, partial, max_parts, tickets, m64,
+                   m32, mnorm2, status, nullptr, 0u, bar, gbase);
 }
 
 // Fallback for very wide rows (D > 8192): same arithmetic, accumulators in shared memory.
@@ -641,17 +681,16 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
 // the packed pairs), one addition of the two, then five shuffle additions: no deeper than the single chain of
 // 8 * ceil(D/256) + 5 operations the selection's error band is derived for.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kScoreThreads)
-score_select(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int n_keep, int nblk,
-             const float* __restrict__ m32, const double* __restrict__ m64, const double* __restrict__ mnorm,
-             float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ tickets,
-             int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(16) uint8_t smem[];
+// The work of one score CTA: block `blk` (kScoreRowsPerCta rows) of chunk b, and the chunk's selection if this CTA hands in
+// the chunk's last block.
+__device__ __forceinline__ void score_role(uint8_t* smem, int b, int blk, const __nv_bfloat16* __restrict__ K, int64_t stride,
+                                           int T, int NA, int D, int n_keep, int nblk, const float* __restrict__ m32,
+                                           const double* __restrict__ m64, const double* __restrict__ mnorm,
+                                           float* __restrict__ s32, float* __restrict__ scores_out,
+                                           uint32_t* __restrict__ tickets, int32_t* __restrict__ keep_idx,
+                                           uint32_t* __restrict__ status) {
   __shared__ uint32_t s_last;
-  dep_wait();
-  dep_release();
   float4* m = reinterpret_cast<float4*>(smem);   // [D/4]; the selection reuses the space afterwards
-  const int b = blockIdx.x / nblk, blk = blockIdx.x - b * nblk;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
   for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
@@ -730,6 +769,114 @@ score_select(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA,
   select_problem<kScoreThreads, false>(smem, b, K, rm, T, NA, D, n_keep, s32, m64, mnorm, keep_idx, status);
 }
 
+__global__ void __launch_bounds__(kScoreThreads)
+score_select(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, int D, int n_keep, int nblk,
+             const float* __restrict__ m32, const double* __restrict__ m64, const double* __restrict__ mnorm,
+             float* __restrict__ s32, float* __restrict__ scores_out, uint32_t* __restrict__ tickets,
+             int32_t* __restrict__ keep_idx, uint32_t* __restrict__ status) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  dep_wait();
+  dep_release();
+  score_role(smem, blockIdx.x / nblk, blockIdx.x % nblk, K, stride, T, NA, D, n_keep, nblk, m32, m64, mnorm, s32, scores_out,
+             tickets, keep_idx, status);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Both passes in one launch.  The anchor pass is bound by instruction issue (fp64), the score pass by memory; run side
+// by side on the same SMs they overlap instead of adding up.  The grid is persistent (as many CTAs as fit the machine);
+// every CTA takes work items from two queues until both are empty:
+//   anchor items (chunk, slice), chunk-major, always available;
+//   score items (chunk, block of rows), chunk-major; the head of that queue is available once its chunk's `ready` word
+//   carries this call's epoch, i.e. once the chunk's last anchor CTA has written the mean anchor.
+// Half of the CTAs prefer score items and half anchor items (each falls back to the other kind), so that both kinds
+// run on every SM; nobody waits while there is work of either kind.  The only wait left: a CTA that has taken a score item
+// of a chunk that is not ready yet (the head moved on between its look and its take) -- bounded, status WK_DEV_TIMEOUT.
+// ------------------------------------------------------------------------------------------------
+struct FusedQueue {
+  uint32_t a_next, s_next, exited, pad;
+};
+
+template <int VPT>
+__global__ void __launch_bounds__(kAnchorThreads, VPT == 1 ? 4 : (VPT == 2 ? 3 : 2))
+compress_fused(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, int T, int NA, int D, int n_keep, int G,
+               int rpp, int parts, int nblk, int layer_ctas, double* __restrict__ partial, int max_parts,
+               uint32_t* __restrict__ tickets_a, uint32_t* __restrict__ tickets_s, uint32_t* ready, FusedQueue* q,
+               uint32_t epoch, double* __restrict__ m64, float* __restrict__ m32, double* __restrict__ mnorm,
+               float* __restrict__ s32, float* __restrict__ scores_out, int32_t* __restrict__ keep_idx,
+               uint32_t* __restrict__ status) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(8) uint64_t bar[2];
+  __shared__ int s_kind, s_item;
+  dep_release();
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    ptx::mbar_init(&bar[0], 1);
+    ptx::mbar_init(&bar[1], 1);
+    ptx::fence_mbar_init();
+  }
+  __syncthreads();
+  const uint32_t a_total = static_cast<uint32_t>(chunks) * parts, s_total = static_cast<uint32_t>(chunks) * nblk;
+  // CTAs that share an SM have block indices layer_ctas apart (one per SM and "layer"): alternate the preference by layer
+  const bool prefer_score = ((blockIdx.x / layer_ctas) & 1) != 0;
+  uint32_t gbase = 0;
+  volatile uint32_t* vq_a = &q->a_next;
+  volatile uint32_t* vq_s = &q->s_next;
+  for (uint32_t idle = 0; idle < (1u << 20);) {
+    if (tid == 0) {
+      int kind = -1, item = 0;      // kind: 0 anchor, 1 score, -1 nothing available now, -2 all work handed out
+      for (int attempt = 0; attempt < 2 && kind < 0; ++attempt) {
+        const bool want_score = (attempt == 0) == prefer_score;
+        if (want_score) {
+          const uint32_t cur = *vq_s;
+          if (cur < s_total && *reinterpret_cast<volatile uint32_t*>(ready + cur / nblk) == epoch) {
+            const uint32_t i = atomicAdd(&q->s_next, 1u);
+            if (i < s_total) { kind = 1; item = static_cast<int>(i); }
+          }
+        } else if (*vq_a < a_total) {
+          const uint32_t i = atomicAdd(&q->a_next, 1u);
+          if (i < a_total) { kind = 0; item = static_cast<int>(i); }
+        }
+      }
+      if (kind < 0 && *vq_a >= a_total && *vq_s >= s_total) kind = -2;
+      if (kind == 1) {
+        // the take may have run ahead of the look into the next chunk: wait for that chunk (rare, short, bounded)
+        const int c = item / nblk;
+        bool ok = false;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+          if (*reinterpret_cast<volatile uint32_t*>(ready + c) == epoch) { ok = true; break; }
+          __nanosleep(100);
+        }
+        if (!ok) { atomicOr(status, WK_DEV_TIMEOUT); kind = -3; }
+        __threadfence();            // the chunk's m32 / m64 are read after the flag
+      }
+      s_kind = kind;
+      s_item = item;
+    }
+    __syncthreads();
+    const int kind = s_kind, item = s_item;
+    __syncthreads();
+    if (kind == -2) break;
+    if (kind == -1) { ++idle; __nanosleep(200); continue; }
+    if (kind == 0) {
+      anchor_role<VPT>(smem, item / parts, item % parts, parts, K, stride, T, D, 1, G, rpp, partial, max_parts, tickets_a,
+                       m64, m32, mnorm, status, ready, epoch, bar, gbase);
+    } else if (kind == 1) {
+      score_role(smem, item / nblk, item % nblk, K, stride, T, NA, D, n_keep, nblk, m32, m64, mnorm, s32, scores_out,
+                 tickets_s, keep_idx, status);
+    }
+    __syncthreads();
+  }
+  // the CTA that leaves last puts the queue back for the next call
+  if (tid == 0) {
+    if (s_kind != -2) atomicOr(status, WK_DEV_TIMEOUT);   // left because nothing became available for far too long
+    if (atomicAdd(&q->exited, 1u) == gridDim.x - 1) {
+      q->a_next = 0u;
+      q->s_next = 0u;
+      q->exited = 0u;
+    }
+  }
+}
+
 // Per-head keys: whole rows again, the dot product and the squared norm taken per 128-column block (lanes 0-15 / 16-31
 // of a 256-column step).  Per lane and head: 8 fused multiply-adds, then 4 shuffle additions -- inside the error band
 // select_pass derives for D = 128.
@@ -799,6 +946,18 @@ void launch_anchor(dim3 grid, size_t smem, cudaStream_t s, const __nv_bfloat16* 
                                                       mnorm2, status);
 }
 
+template <int VPT>
+void launch_fused(unsigned grid, size_t smem, cudaStream_t s, const __nv_bfloat16* K, int64_t stride, int chunks, int T, int NA,
+                  int D, int n_keep, int G, int rpp, int parts, int nblk, int layer_ctas, double* partial, int max_parts,
+                  uint32_t* tickets_a, uint32_t* tickets_s, uint32_t* ready, FusedQueue* q, uint32_t epoch, double* m64,
+                  float* m32, double* mnorm, float* s32, float* scores_out, int32_t* keep_idx, uint32_t* status) {
+  if (smem > 48 * 1024)
+    cudaFuncSetAttribute(compress_fused<VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  compress_fused<VPT><<<grid, kAnchorThreads, smem, s>>>(K, stride, chunks, T, NA, D, n_keep, G, rpp, parts, nblk, layer_ctas,
+                                                         partial, max_parts, tickets_a, tickets_s, ready, q, epoch, m64, m32,
+                                                         mnorm, s32, scores_out, keep_idx, status);
+}
+
 }  // namespace
 
 wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, int chunks, int32_t* keep_idx,
@@ -844,9 +1003,33 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       int rpp = (T + parts - 1) / parts;
       rpp = (rpp + G - 1) / G * G;            // whole groups, so that only a chunk's last slice has a short group
       parts = (T + rpp - 1) / rpp;
+      const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 1 .. 4 for DF <= 8192
+      if (!per_head && n_keep > 0 && n_keep < NA) {
+        // whole-key scoring with a real selection: both passes in one launch
+        const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
+        const size_t smem_s = smem_sel > smem_m ? smem_sel : smem_m;
+        const size_t smem_f = smem_a > smem_s ? smem_a : smem_s;
+        // persistent grid: what fits the machine at this shared-memory size (the same bound the slices were cut for)
+        int per_sm_f = static_cast<int>((220 * 1024) / (smem_f + 2048));
+        const int by_regs_f = vpt == 1 ? 4 : (vpt == 2 ? 3 : 2);
+        if (per_sm_f > by_regs_f) per_sm_f = by_regs_f;
+        if (per_sm_f < 1) per_sm_f = 1;
+        unsigned grid_f = static_cast<unsigned>(ctx->sm_count * per_sm_f);
+        const unsigned items = static_cast<unsigned>(chunks) * static_cast<unsigned>(parts + nblk);
+        if (grid_f > items) grid_f = items;
+        uint32_t* ready = tickets + 2 * ctx->max_batch;
+        FusedQueue* q = reinterpret_cast<FusedQueue*>(tickets + 3 * ctx->max_batch);
+        const uint32_t epoch = ++ctx->compress_epoch;
+#define WK_FUSED(V) launch_fused<V>(grid_f, smem_f, s, K, stride, chunks, T, NA, DF, n_keep, G, rpp, parts, nblk, ctx->sm_count, partial, max_parts, tickets, tickets + ctx->max_batch, ready, q, epoch, m64, m32, mnorm, s32, scores_out, keep_idx, ctx->status_dev)
+        if (vpt <= 1) WK_FUSED(1);
+        else if (vpt == 2) WK_FUSED(2);
+        else if (vpt == 3) WK_FUSED(3);
+        else WK_FUSED(4);
+#undef WK_FUSED
+        return after_launch(ctx);
+      }
       const dim3 grid(parts, chunks);
       const int hs = per_head ? H : 1;
-      const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 1 .. 4 for DF <= 8192
 #define WK_ANCHOR(V) launch_anchor<V>(grid, smem_a, s, K, stride, T, DF, hs, G, rpp, partial, max_parts, tickets, m64, m32, mnorm, ctx->status_dev)
       if (vpt <= 1) WK_ANCHOR(1);
       else if (vpt == 2) WK_ANCHOR(2);

@@ -78,6 +78,7 @@ struct wk_ctx {
   size_t tmap_cache_next = 0;
   // per-context (hence per-device) one-time kernel attributes: opt-ins to large dynamic shared memory
   bool attn_attr_set = false;
+  uint32_t compress_epoch = 0;   // call counter of the one-launch compression: its `ready` words compare against it
   // diagnostics
   int32_t last_cuda_error = 0;
   int64_t launches = 0;
