@@ -20,6 +20,7 @@
  *   - Ownership: the caller owns every device buffer, including pool storage and scratch (sizes come
  *     from wk_pool_bytes / wk_scratch_bytes; the context only keeps host-side bookkeeping and tensor
  *     maps).  No call allocates device memory.  One context may be used by one host thread at a time.
+ *   - The calls of one context share its scratch buffer: enqueue them on one stream, or order the streams yourself.
  *   - There is no CPU fallback: without a CUDA device of compute capability 10.x, wk_create fails.
  */
 #ifndef WK_H_
@@ -168,7 +169,9 @@ wk_status wk_pool_load_host(wk_ctx* ctx, int32_t layer0, int32_t n, const void* 
  * rotation angle, each divided by its maximum over the stored chunks, summed.  Writes the min(k, M)
  * slots with the smallest distance, ties to the lowest slot, in rank order.
  *   slots_out_dev [max_k] int32 (entries past the count are set to -1); dist_out_dev [max_k] fp64 or NULL
- *   n_out_host    the count min(k, M), known on the host
+ *   n_out_host    the count min(k, M), known on the host (M counts the valid slots)
+ * A stored or current pose with a NaN/Inf component is not a candidate: WK_DEV_NONFINITE is set and the places it would
+ * have taken stay -1.
  * Errors: WK_ERR_SHAPE (k > max_k or k < 0), WK_ERR_ARG, WK_ERR_UNBOUND. */
 wk_status wk_retrieve(wk_ctx* ctx, const float* cur_pose_host, int32_t k, int32_t* slots_out_dev,
                       double* dist_out_dev, int32_t* n_out_host, void* stream);
@@ -187,8 +190,11 @@ wk_status wk_retrieve_query(wk_ctx* ctx, int32_t layer, const void* Q, int32_t l
  * wk_retrieve: squared-L2 translation distance and geodesic rotation angle, each divided by its maximum over the valid
  * candidates, summed, in fp64; the min(k, valid candidates) smallest win, ties to the lowest index, rank order).  For
  * candidate sets far beyond a pool's slot table (the paper's pools hold 10^2..10^3 chunks; this call is what makes
- * "GB/s of retrieval" measurable at 2^16..2^24 poses).  The poses are read twice: both maxima must be known before any
- * distance can be formed.
+ * "GB/s of retrieval" measurable at 2^16..2^24 poses).  The poses are read once: a sampled set of k real candidates
+ * rules most others out before the two maxima are known (a candidate that k others beat for every possible pair of
+ * maxima is not among the k best); the few that remain are ranked exactly afterwards.  Pose sets where nothing can be
+ * ruled out (e.g. all rotations equal) are read a second time instead; the result is the same either way.  A pose with
+ * a NaN/Inf component is never a candidate and sets WK_DEV_NONFINITE.
  *   poses_dev [n][8] fp32 (tx ty tz _ qw qx qy qz), 16-byte aligned; valid_dev [n] int32 or NULL (all valid);
  *   cur_pose_host [8]; ids_out_dev [out_capacity] int32 (-1 past the count); dist_out_dev [out_capacity] fp64 or NULL;
  *   scratch_dev: wk_retrieve_scan_scratch_bytes() bytes, 16-byte aligned, caller-owned, contents irrelevant on entry.
@@ -213,6 +219,7 @@ wk_status wk_retrieve_scan(wk_ctx* ctx, const float* poses_dev, const int32_t* v
  * stream capture.  All calls on a device share the one array: two calls whose kernels may overlap on the GPU
  * (different streams) race on it; calls on one stream are safe.  Nothing in the array has to start at zero: every
  * entry a call reads it has written first.  Calls no cudaMalloc/cudaFree and no allocating library routine.
+ * A pose with a NaN/Inf component is not a candidate (there is no status word to report it through here).
  * Errors: WK_ERR_ARG, WK_ERR_SHAPE, WK_ERR_NO_DEVICE, WK_ERR_CUDA. */
 wk_status wk_retrieve_noalloc(const float* poses_dev, const int32_t* valid_dev, int32_t n_slots,
                               const float* cur_pose_host, int32_t k, int32_t max_k, int32_t* slots_out_dev,

@@ -432,14 +432,17 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
     return !(lb > s_tau_hi) || t > 3.0e38f;   // an fp32 overflow of t says nothing about t / mt
   };
   // exact distance of one candidate, the arithmetic of retrieve_kernel
-  auto exact = [&](int32_t i, double tau) {
-    const Cand c = candidate(__ldg(poses + 2 * static_cast<int64_t>(i)), __ldg(poses + 2 * static_cast<int64_t>(i) + 1), cur.v);
+  auto exact_of = [&](const float4 pa, const float4 pb, int32_t i, double tau) {
+    const Cand c = candidate(pa, pb, cur.v);
     if (!isfinite(c.t) || !isfinite(c.adot)) return;         // not a candidate (reported by the pass that read it first)
     const double rot = 2.0 * acos(fmin(1.0, c.adot));
     const double ta = mt > 0.0 ? c.t / mt : 0.0;
     const double rb = mr > 0.0 ? rot / mr : 0.0;
     const double dist = ta + rb;
     if (dist <= tau) top.push(dist, i);
+  };
+  auto exact = [&](int32_t i, double tau) {
+    exact_of(__ldg(poses + 2 * static_cast<int64_t>(i)), __ldg(poses + 2 * static_cast<int64_t>(i) + 1), i, tau);
   };
   if (threadIdx.x == 0) s_npend[0] = s_npend[1] = 0;
   refresh();
@@ -495,6 +498,17 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
         a[u] = __ldg(poses + 2 * static_cast<int64_t>(ci[u]));
         b[u] = __ldg(poses + 2 * static_cast<int64_t>(ci[u]) + 1);
       }
+    }
+    if (listed) {
+      // listed candidates have passed a sharper test already: straight to the exact distance, one entry per thread
+      // and list check (the list has room for one push per thread between checks)
+#pragma unroll
+      for (int u = 0; u < kScanUnroll; ++u) {
+        if ((r * kScanUnroll + u) * kSelThreads * gridDim.x + blockIdx.x >= n) break;   // same for the whole block
+        if (live[u]) exact_of(a[u], b[u], ci[u], s_tau);
+        if (top.round_end()) top.compact();
+      }
+      continue;
     }
 #pragma unroll
     for (int u = 0; u < kScanUnroll; ++u)
