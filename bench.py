@@ -586,6 +586,7 @@ def run_ours(args, w: wi.Workload):
     rank, local_rank, world = dist_env()
     if world > 1:
         import torch.distributed as dist
+        os.environ.setdefault("NCCL_DEBUG", "INFO")   # the communicator log (stderr) shows the ranks that joined
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     from paper_2605_22718_b200.build import build_all
