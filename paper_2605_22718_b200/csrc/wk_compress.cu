@@ -683,18 +683,22 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
 // ------------------------------------------------------------------------------------------------
 // The work of one score CTA: block `blk` (kScoreRowsPerCta rows) of chunk b, and the chunk's selection if this CTA hands in
 // the chunk's last block.
-__device__ __forceinline__ void score_role(uint8_t* smem, int b, int blk, const __nv_bfloat16* __restrict__ K, int64_t stride,
+__device__ __forceinline__ bool score_role(uint8_t* smem, int b, int blk, const __nv_bfloat16* __restrict__ K, int64_t stride,
                                            int T, int NA, int D, int n_keep, int nblk, const float* __restrict__ m32,
                                            const double* __restrict__ m64, const double* __restrict__ mnorm,
                                            float* __restrict__ s32, float* __restrict__ scores_out,
                                            uint32_t* __restrict__ tickets, int32_t* __restrict__ keep_idx,
-                                           uint32_t* __restrict__ status) {
+                                           uint32_t* __restrict__ status, bool m_staged = false) {
+  // m_staged: the chunk's m32 is in shared memory already (the CTA's previous item was a block of the same chunk).
+  // Returns true if shared memory still holds it on return, false if the selection has used the space.
   __shared__ uint32_t s_last;
   float4* m = reinterpret_cast<float4*>(smem);   // [D/4]; the selection reuses the space afterwards
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
-  for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
-  __syncthreads();
+  if (!m_staged) {
+    const float4* msrc = reinterpret_cast<const float4*>(m32 + static_cast<int64_t>(b) * D);
+    for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
+    __syncthreads();
+  }
   const int vecs = D >> 3;
   const int j0 = blk * kScoreRowsPerCta;
   const int j1 = min(NA, j0 + kScoreRowsPerCta);
@@ -756,17 +760,18 @@ __device__ __forceinline__ void score_role(uint8_t* smem, int b, int blk, const 
       if (scores_out) scores_out[static_cast<int64_t>(b) * NA + jj] = sc;
     }
   }
-  if (keep_idx == nullptr) return;   // scores only
+  if (keep_idx == nullptr) return true;   // scores only
   // hand in this block of rows; the CTA that completes the problem selects
   __threadfence();
   __syncthreads();
   if (tid == 0) s_last = (atomicAdd(&tickets[b], 1u) == static_cast<uint32_t>(nblk - 1)) ? 1u : 0u;
   __syncthreads();
-  if (!s_last) return;
+  if (!s_last) return true;
   __threadfence();
   if (tid == 0) tickets[b] = 0;   // ready for the next call
   const RowMap rm{stride, D, 1};
   select_problem<kScoreThreads, false>(smem, b, K, rm, T, NA, D, n_keep, s32, m64, mnorm, keep_idx, status);
+  return false;
 }
 
 __global__ void __launch_bounds__(kScoreThreads)
@@ -819,6 +824,7 @@ compress_fused(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, 
   // CTAs that share an SM have block indices layer_ctas apart (one per SM and "layer"): alternate the preference by layer
   const bool prefer_score = ((blockIdx.x / layer_ctas) & 1) != 0;
   uint32_t gbase = 0;
+  int staged_chunk = -1;   // chunk whose m32 this CTA's shared memory holds, if any
   volatile uint32_t* vq_a = &q->a_next;
   volatile uint32_t* vq_s = &q->s_next;
   for (uint32_t idle = 0; idle < (1u << 20);) {
@@ -858,11 +864,14 @@ compress_fused(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, 
     if (kind == -2) break;
     if (kind == -1) { ++idle; __nanosleep(200); continue; }
     if (kind == 0) {
+      staged_chunk = -1;
       anchor_role<VPT>(smem, item / parts, item % parts, parts, K, stride, T, D, 1, G, rpp, partial, max_parts, tickets_a,
                        m64, m32, mnorm, status, ready, epoch, bar, gbase);
     } else if (kind == 1) {
-      score_role(smem, item / nblk, item % nblk, K, stride, T, NA, D, n_keep, nblk, m32, m64, mnorm, s32, scores_out,
-                 tickets_s, keep_idx, status);
+      const int c = item / nblk;
+      const bool kept = score_role(smem, c, item % nblk, K, stride, T, NA, D, n_keep, nblk, m32, m64, mnorm, s32,
+                                   scores_out, tickets_s, keep_idx, status, staged_chunk == c);
+      staged_chunk = kept ? c : -1;
     }
     __syncthreads();
   }
@@ -996,7 +1005,9 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       int per_sm = static_cast<int>((220 * 1024) / (smem_a + 1024));
       const int by_regs = DF > 2048 ? 2 : 4;
       if (per_sm > by_regs) per_sm = by_regs;
-      int parts = ctx->sm_count * (per_sm < 1 ? 1 : per_sm) / chunks;
+      // about a third more slices than CTA slots (measured: shorter items even out the end of the launch; flat between
+      // 1.2 and 1.6 slots' worth at both model shapes)
+      int parts = (ctx->sm_count * (per_sm < 1 ? 1 : per_sm) * 27 / 20 + chunks - 1) / chunks;
       if (parts < 1) parts = 1;
       if (parts > max_parts) parts = max_parts;
       if (parts > (T + G - 1) / G) parts = (T + G - 1) / G;
