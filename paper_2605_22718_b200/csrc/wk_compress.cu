@@ -4,18 +4,21 @@
 // The mean over anchors is pulled inside the dot product: s_j = (k_j . m) / |k_j| with
 // m = (1/T) sum_i a_i / |a_i|, so a chunk is read exactly once (3T*D bf16) instead of T^2 times.
 //
-//   anchor_pass   reads the T anchor rows once: groups of rows arrive in shared memory by bulk copy (double-buffered),
-//                 a warp takes the fp64 norm of a row, then every thread adds a_i / |a_i| for the columns it owns, in
-//                 fp64, over the rows of the group.  A CTA covers one slice of one problem's rows; the last CTA of a
-//                 problem (atomic ticket, nobody waits) adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|^2
+//   anchor_rows   reads the T anchor rows once.  A row is shared by a set of warps; each lane converts its share to fp64
+//                 once and keeps it in registers: fp64 squared norm (warp sum, plus an exchange between the set's warps),
+//                 then a_i / |a_i| is added to the lane's own fp64 column sums.  Every CTA takes an equal run of the
+//                 rows of all chunks and hands in one slice of column sums per chunk it touches; the last CTA of a
+//                 chunk (atomic ticket, nobody waits) adds the slices in a fixed order -> m64, m32 = fp32(m64), |m|^2
 //   score_select  reads the (F-1)T non-anchor rows once: fp32 dot with the shared-memory-staged m32 and fp32 norm,
 //                 warp-shuffle reductions -> s32.  The CTA that finishes a problem's last rows (ticket again) runs that
 //                 problem's selection while the other CTAs are still streaming later problems:
 //   selection     the n_keep-th smallest s32 (radix select) is the threshold; tokens further than a proved fp32 error
 //                 band from it are decided at once, the few inside the band are re-scored in fp64 against m64 and
 //                 ranked exactly by (score, index); emits the ascending index list
-// Per-head keys (one keep-set per head) use the same anchor_pass with per-head norms, then head_score and a
-// selection launch of its own (n_heads problems per chunk).
+//   compress_fused  wide whole-token rows (more than 2,048 columns): both passes in one persistent launch, anchor CTAs
+//                 (rows staged in shared memory, anchor_role) and score CTAs side by side on every SM
+// Per-head keys (one keep-set per head) use anchor_rows with per-head norms, then head_score and a selection launch of
+// its own (n_heads problems per chunk).
 //
 // The selection is therefore decided in fp64 wherever fp32 could not decide it, and is reproducible
 // run to run (no floating-point atomics anywhere).
@@ -80,20 +83,26 @@ __device__ __forceinline__ float half_warp_sum(float v) {
 // 1023 - 127 = 896 and the seven mantissa bits at the top of the fraction -- two or three integer operations where the
 // conversion instruction runs at a quarter of the fp64 multiply-add rate.  w holds two bf16 values (low and high half).
 // An exponent field of 0 (zero, subnormal) comes out as a number below 2^-126 and a field of 255 (Inf, NaN) as one of at
-// least 2^128: anchor_pass looks at every row's squared norm, and a group of rows with a norm outside [2^-40, 2^125] is
+// least 2^128: anchor_role looks at every row's squared norm, and a group of rows with a norm outside [2^-80, 2^250] is
 // redone with the exact conversions below.  Inside that range a mis-read zero or subnormal moves a column sum by less
-// than 2^-126 * 2^40 = 2^-86 per row, far below the rounding of the fp64 sums themselves.
-__device__ __forceinline__ double bf16_lo_abs_fast(uint32_t w) {
-  return __hiloint2double(static_cast<int>(((w & 0x7FFFu) << 13) + 0x38000000u), 0);
+// than 2^-126 * 2^40 = 2^-86 per row, far below the rounding of the fp64 sums themselves.  (anchor_rows converts every
+// element with the conversion instruction and needs none of this.)
+// One widening multiply-add builds the whole double: the 15 magnitude bits, moved to the top of a 32-bit word, times
+// 2^28 land on bits 59..45 of the 64-bit product (low word zero), and the addend carries the re-biased exponent.
+__device__ __forceinline__ double mad_wide_f64(uint32_t a, uint32_t b) {
+  uint64_t r;
+  asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"(0x3800000000000000ull));
+  return __longlong_as_double(static_cast<long long>(r));
 }
-__device__ __forceinline__ double bf16_hi_abs_fast(uint32_t w) {
-  return __hiloint2double(static_cast<int>(__umulhi(w & 0x7FFF0000u, 0x20000000u) + 0x38000000u), 0);
-}
+__device__ __forceinline__ double bf16_lo_abs_fast(uint32_t w) { return mad_wide_f64(w << 17, 1u << 28); }
+__device__ __forceinline__ double bf16_hi_abs_fast(uint32_t w) { return mad_wide_f64(w & 0x7FFF0000u, 1u << 29); }
 __device__ __forceinline__ double bf16_lo_fast(uint32_t w) {
-  return __hiloint2double(static_cast<int>((((w & 0x7FFFu) << 13) + 0x38000000u) | ((w << 16) & 0x80000000u)), 0);
+  const double d = bf16_lo_abs_fast(w);
+  return __hiloint2double(__double2hiint(d) | static_cast<int>((w << 16) & 0x80000000u), __double2loint(d));
 }
 __device__ __forceinline__ double bf16_hi_fast(uint32_t w) {
-  return __hiloint2double(static_cast<int>((__umulhi(w & 0x7FFF0000u, 0x20000000u) + 0x38000000u) | (w & 0x80000000u)), 0);
+  const double d = bf16_hi_abs_fast(w);
+  return __hiloint2double(__double2hiint(d) | static_cast<int>(w & 0x80000000u), __double2loint(d));
 }
 template <bool kExact> __device__ __forceinline__ double bf16_lo(uint32_t w) {
   return kExact ? static_cast<double>(__uint_as_float(w << 16)) : bf16_lo_fast(w);
@@ -109,86 +118,60 @@ template <bool kExact> __device__ __forceinline__ double bf16_hi_abs(uint32_t w)
 }
 
 // ------------------------------------------------------------------------------------------------
-// anchor pass.  grid = (parts, chunks), 256 threads.  CTA (part, chunk) owns rows [part * rpp, (part + 1) * rpp) of
-// the chunk's anchor frame and walks them in groups of G rows:
+// Staged anchor role of the one-launch kernel (whole-token keys).  Work item (part, chunk) owns rows
+// [part * rpp, (part + 1) * rpp) of the chunk's anchor frame and walks them in groups of G rows:
 //   thread 0 keeps one bulk copy (the next group's G contiguous rows) in flight into the other half of the row buffer;
 //   phase 1: the 8 warps share the group's rows (8 / G column segments per row): fp64 squared norms from shared memory
-//            -> 1/|a| (0 for a zero key); with per-head keys (hs = n_heads) one norm per 128-column block, reduced
-//            within 16 lanes;
+//            -> 1/|a| (0 for a zero key);
 //   phase 2: thread t owns the 16-byte column groups t, t + 256, ...: a_i[c] / |a_i| is added over the rows of the group.
 // The CTA writes its column sums as one slice; the last CTA of the chunk adds the slices in slice order and writes
-// m64, m32 = fp32(m64) and |m|^2 (per head with per-head keys).  VPT = 16-byte column groups per thread = ceil(D / 2048).
+// m64, m32 = fp32(m64) and |m|^2.  VPT = 16-byte column groups per thread = ceil(D / 2048).
 // ------------------------------------------------------------------------------------------------
 constexpr int kAnchorThreads = 256;
 constexpr int kAnchorWarps = kAnchorThreads / 32;
 constexpr double kNorm2Lo = 8.2718061255302767e-25;    // 2^-80: squared norm below which a row is redone exactly
 constexpr double kNorm2Hi = 1.8092513943330656e+75;    // 2^250: likewise above
 
-// squared norms of the group's rows: warp -> (row, column segment); n2_s[row][seg] (whole keys) or n2_s[row][head]
+// squared norms of the group's rows: warp -> (row, column segment); n2_s[row][seg]
 template <bool kExact>
 __device__ __forceinline__ void group_norms(const uint8_t* buf, size_t row_bytes, int rows, int nseg, int seg_vecs, int vecs,
-                                            int hs, int n2_pitch, double* n2_s) {
+                                            double* n2_s) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = warp / nseg, seg = warp - r * nseg;
   if (r >= rows) return;
   const uint4* row = reinterpret_cast<const uint4*>(buf + r * row_bytes);
   const int v_begin = seg * seg_vecs, v_end = min(vecs, v_begin + seg_vecs);
-  if (hs == 1) {
-    double n2a = 0.0, n2b = 0.0;
-    for (int v = v_begin + lane; v < v_end; v += 32) {
-      const uint4 q = row[v];
-      const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-      // three of the eight conversions go to the conversion unit, five to the integer pipe: both stay busy
-      {
-        const double x0 = bf16_lo_abs<true>(w[0]), x1 = bf16_hi_abs<kExact>(w[0]);
-        const double x2 = bf16_lo_abs<kExact>(w[1]), x3 = bf16_hi_abs<true>(w[1]);
-        const double x4 = bf16_lo_abs<kExact>(w[2]), x5 = bf16_hi_abs<kExact>(w[2]);
-        const double x6 = bf16_lo_abs<true>(w[3]), x7 = bf16_hi_abs<kExact>(w[3]);
-        n2a = fma(x0, x0, n2a); n2b = fma(x1, x1, n2b);
-        n2a = fma(x2, x2, n2a); n2b = fma(x3, x3, n2b);
-        n2a = fma(x4, x4, n2a); n2b = fma(x5, x5, n2b);
-        n2a = fma(x6, x6, n2a); n2b = fma(x7, x7, n2b);
-      }
-    }
-    const double n2 = warp_sum(n2a + n2b);
-    if (lane == 0) n2_s[r * n2_pitch + seg] = n2;
-  } else {
-    for (int v = v_begin + lane; v - lane < v_end; v += 32) {   // a 32-lane step covers two heads: lanes 0-15 / 16-31
-      double n2a = 0.0, n2b = 0.0;
-      if (v < v_end) {
-        const uint4 q = row[v];
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-        {
-          const double x0 = bf16_lo_abs<true>(w[0]), x1 = bf16_hi_abs<kExact>(w[0]);
-          const double x2 = bf16_lo_abs<kExact>(w[1]), x3 = bf16_hi_abs<true>(w[1]);
-          const double x4 = bf16_lo_abs<kExact>(w[2]), x5 = bf16_hi_abs<kExact>(w[2]);
-          const double x6 = bf16_lo_abs<true>(w[3]), x7 = bf16_hi_abs<kExact>(w[3]);
-          n2a = fma(x0, x0, n2a); n2b = fma(x1, x1, n2b);
-          n2a = fma(x2, x2, n2a); n2b = fma(x3, x3, n2b);
-          n2a = fma(x4, x4, n2a); n2b = fma(x5, x5, n2b);
-          n2a = fma(x6, x6, n2a); n2b = fma(x7, x7, n2b);
-        }
-      }
-      const double n2 = half_warp_sum(n2a + n2b);
-      if ((lane & 15) == 0 && v < v_end) n2_s[r * n2_pitch + (v >> 4)] = n2;
-    }
+  double n2a = 0.0, n2b = 0.0;
+  for (int v = v_begin + lane; v < v_end; v += 32) {
+    const uint4 q = row[v];
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+    // three of the eight conversions go to the conversion unit, five to the integer pipe: both stay busy
+    const double x0 = bf16_lo_abs<true>(w[0]), x1 = bf16_hi_abs<kExact>(w[0]);
+    const double x2 = bf16_lo_abs<kExact>(w[1]), x3 = bf16_hi_abs<true>(w[1]);
+    const double x4 = bf16_lo_abs<kExact>(w[2]), x5 = bf16_hi_abs<kExact>(w[2]);
+    const double x6 = bf16_lo_abs<true>(w[3]), x7 = bf16_hi_abs<kExact>(w[3]);
+    n2a = fma(x0, x0, n2a); n2b = fma(x1, x1, n2b);
+    n2a = fma(x2, x2, n2a); n2b = fma(x3, x3, n2b);
+    n2a = fma(x4, x4, n2a); n2b = fma(x5, x5, n2b);
+    n2a = fma(x6, x6, n2a); n2b = fma(x7, x7, n2b);
   }
+  const double n2 = warp_sum(n2a + n2b);
+  if (lane == 0) n2_s[r * nseg + seg] = n2;
 }
 
 // column sums of a / |a| over the rows of the group, for the 16-byte column groups this thread owns (t, t + 256, ...)
 template <int VPT, bool kExact>
-__device__ __forceinline__ void group_accumulate(const uint8_t* buf, size_t row_bytes, int rows, int vecs, int hs,
+__device__ __forceinline__ void group_accumulate(const uint8_t* buf, size_t row_bytes, int rows, int vecs,
                                                  const double* inv_s, double (&acc)[8 * VPT]) {
   const int tid = threadIdx.x;
   for (int r = 0; r < rows; ++r) {
     const uint4* row = reinterpret_cast<const uint4*>(buf + r * row_bytes);
-    const double* inv = inv_s + r * hs;
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
       const int vec = tid + i * kAnchorThreads;
       if (vec < vecs) {
         const uint4 q = row[vec];
-        const double sc = inv[hs == 1 ? 0 : (vec >> 4)];
+        const double sc = inv_s[r];
         double* a = acc + 8 * i;
         a[0] = fma(bf16_lo<true>(q.x), sc, a[0]);
         a[1] = fma(bf16_hi<kExact>(q.x), sc, a[1]);
@@ -203,26 +186,102 @@ __device__ __forceinline__ void group_accumulate(const uint8_t* buf, size_t row_
   }
 }
 
+// After a CTA has written its slice of chunk b: the last CTA of the chunk (an atomic ticket decides) adds the slices in
+// slice order and writes m64, m32 = fp32(m64) and |m|^2 (per head with per-head keys).  Called by every thread of the CTA.
+__device__ __forceinline__ void anchor_finish(int b, int parts, int T, int D, int hs, const double* __restrict__ partial,
+                                              int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
+                                              float* __restrict__ m32, double* __restrict__ mnorm2, uint32_t* ready,
+                                              uint32_t epoch) {
+  __shared__ uint32_t s_flag;
+  __shared__ double red[32];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nthr = blockDim.x, nwarps = nthr >> 5;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_flag = (atomicAdd(&tickets[b], 1u) == static_cast<uint32_t>(parts - 1)) ? 1u : 0u;
+  __syncthreads();
+  if (!s_flag) return;
+  // ---- last CTA of the chunk: add the slices in slice order.  Thread t owns column pairs t, t + 256, ...; eight
+  // slices' worth of loads are in flight before the first addition.
+  __threadfence();
+  const double* pb = partial + static_cast<int64_t>(b) * max_parts * D;
+  const double inv_T = 1.0 / static_cast<double>(T);
+  const int pairs = D >> 1;
+  double nn_all = 0.0;
+  for (int c0 = 0; c0 < pairs; c0 += nthr) {   // uniform trip count: the per-head sums use block barriers
+    const int c = c0 + tid;
+    double t0 = 0.0, t1 = 0.0;
+    if (c < pairs) {
+      for (int p0 = 0; p0 < parts; p0 += 8) {
+        double2 v[8];
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp)
+          v[pp] = p0 + pp < parts ? __ldcg(reinterpret_cast<const double2*>(pb + static_cast<int64_t>(p0 + pp) * D) + c)
+                                  : make_double2(0.0, 0.0);
+#pragma unroll
+        for (int pp = 0; pp < 8; ++pp) {
+          t0 += v[pp].x;
+          t1 += v[pp].y;
+        }
+      }
+      t0 *= inv_T;
+      t1 *= inv_T;
+      reinterpret_cast<double2*>(m64 + static_cast<int64_t>(b) * D)[c] = make_double2(t0, t1);
+      reinterpret_cast<float2*>(m32 + static_cast<int64_t>(b) * D)[c] =
+          make_float2(static_cast<float>(t0), static_cast<float>(t1));
+    }
+    const double nn = fma(t0, t0, t1 * t1);
+    if (hs == 1) {
+      nn_all += nn;
+    } else {
+      // 64 column pairs per head: warps 2j and 2j + 1 of this step hold head c0 / 64 + j
+      const double wsum = warp_sum(nn);
+      __syncthreads();
+      if (lane == 0) red[warp] = wsum;
+      __syncthreads();
+      const int head = (c0 >> 6) + tid;
+      if (tid < nwarps / 2 && head < hs)
+        mnorm2[(static_cast<int64_t>(b) * hs + head) * kMaxNormParts] = red[2 * tid] + red[2 * tid + 1];
+    }
+  }
+  if (hs == 1) {
+    const double wsum = warp_sum(nn_all);
+    if (lane == 0) red[warp] = wsum;
+    __syncthreads();
+    if (tid == 0) {
+      double t = 0.0;
+      for (int w = 0; w < nwarps; ++w) t += red[w];
+      mnorm2[static_cast<int64_t>(b) * kMaxNormParts] = t;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    tickets[b] = 0;   // ready for the next call
+    if (ready) {
+      __threadfence();                                   // m64 / m32 / |m|^2 of every thread are out before the flag
+      *reinterpret_cast<volatile uint32_t*>(ready + b) = epoch;
+    }
+  }
+}
+
 // The work of one anchor CTA (slice `part` of `parts` of chunk b).  `ready` (may be null): a word per chunk that the last
 // CTA of the chunk sets to `epoch` once m64 / m32 / |m|^2 are written, for score CTAs of the same launch to poll.
 template <int VPT>
 __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int parts, const __nv_bfloat16* __restrict__ K,
-                                            int64_t stride, int T, int D, int hs, int G, int rpp,
+                                            int64_t stride, int T, int D, int G, int rpp,
                                             double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets,
                                             double* __restrict__ m64, float* __restrict__ m32, double* __restrict__ mnorm2,
                                             uint32_t* __restrict__ status, uint32_t* ready, uint32_t epoch,
                                             uint64_t* bar, uint32_t& gbase) {
   // bar[2]: the caller's two mbarriers (initialised once per CTA, count 1); gbase: bulk copies this CTA has waited for so
   // far -- copy number n lands in buffer n & 1 and completes phase n >> 1 of barrier n & 1
-  __shared__ uint32_t s_flag;
-  __shared__ double red[kAnchorWarps];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const size_t row_bytes = static_cast<size_t>(D) * 2;
   const int nseg = kAnchorWarps / G;                                        // column segments per row in phase 1
-  const int n2_pitch = hs == 1 ? nseg : hs;
   uint8_t* rows_s = smem;                                                   // [2][G][D] bf16
-  double* inv_s = reinterpret_cast<double*>(smem + 2 * G * row_bytes);      // [G][hs]
-  double* n2_s = inv_s + G * hs;                                            // [G][n2_pitch]
+  double* inv_s = reinterpret_cast<double*>(smem + 2 * G * row_bytes);      // [G]
+  double* n2_s = inv_s + G;                                                 // [G][nseg]
   const int r0 = min(T, part * rpp), r1 = min(T, r0 + rpp);
   const int n_groups = (r1 - r0 + G - 1) / G;
   const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride;
@@ -258,13 +317,13 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
     const int rows = min(G, r1 - (r0 + g * G));
     const uint8_t* buf = rows_s + (n_cur & 1) * G * row_bytes;
     // ---- phase 1: norms (integer-pipe conversions; redone exactly when a norm falls outside the safe range)
-    group_norms<false>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
+    group_norms<false>(buf, row_bytes, rows, nseg, seg_vecs, vecs, n2_s);
     bool redo = false;
-    if (hs == 1 && nseg == 1) {
+    if (nseg == 1) {
       // one warp holds a whole row's squared norm: its first lane finishes the row on the spot, so that the eight
       // reciprocal square roots run side by side and one barrier (the vote below) ends the phase
       if (warp < rows && lane == 0) {
-        const double n2 = n2_s[warp * n2_pitch];
+        const double n2 = n2_s[warp];
         inv_s[warp] = n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);
         redo = !(n2 >= kNorm2Lo && n2 <= kNorm2Hi);
       }
@@ -272,26 +331,24 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
       __syncthreads();
     }
     auto finish_norms = [&](bool check) {
-      for (int i = tid; i < rows * hs; i += kAnchorThreads) {
-        const int r = i / hs, h = i - r * hs;
+      for (int r = tid; r < rows; r += kAnchorThreads) {
         double n2 = 0.0;
-        if (hs == 1) for (int sg = 0; sg < nseg; ++sg) n2 += n2_s[r * n2_pitch + sg];
-        else n2 = n2_s[r * n2_pitch + h];
-        inv_s[i] = n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);   // zero key: cosine 0; a NaN norm stays NaN
+        for (int sg = 0; sg < nseg; ++sg) n2 += n2_s[r * nseg + sg];
+        inv_s[r] = n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);   // zero key: cosine 0; a NaN norm stays NaN
         if (check) redo = redo || !(n2 >= kNorm2Lo && n2 <= kNorm2Hi);
       }
     };
-    if (!(hs == 1 && nseg == 1)) finish_norms(true);
+    if (nseg != 1) finish_norms(true);
     const bool exact = __syncthreads_or(redo) != 0;
     if (exact) {
-      group_norms<true>(buf, row_bytes, rows, nseg, seg_vecs, vecs, hs, n2_pitch, n2_s);
+      group_norms<true>(buf, row_bytes, rows, nseg, seg_vecs, vecs, n2_s);
       __syncthreads();
       finish_norms(false);
       __syncthreads();
-      group_accumulate<VPT, true>(buf, row_bytes, rows, vecs, hs, inv_s, acc);
+      group_accumulate<VPT, true>(buf, row_bytes, rows, vecs, inv_s, acc);
     } else {
       // ---- phase 2
-      group_accumulate<VPT, false>(buf, row_bytes, rows, vecs, hs, inv_s, acc);
+      group_accumulate<VPT, false>(buf, row_bytes, rows, vecs, inv_s, acc);
     }
     __syncthreads();   // the group's buffer, inv_s and n2_s may be overwritten from here on
   }
@@ -314,92 +371,192 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
         __stcg(reinterpret_cast<double2*>(my + 8 * vec) + e, make_double2(acc[8 * i + 2 * e], acc[8 * i + 2 * e + 1]));
     }
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_flag = (atomicAdd(&tickets[b], 1u) == static_cast<uint32_t>(parts - 1)) ? 1u : 0u;
-  __syncthreads();
-  if (!s_flag) return;
-  // ---- last CTA of the chunk: add the slices in slice order.  Thread t owns column pairs t, t + 256, ...; eight
-  // slices' worth of loads are in flight before the first addition.
-  __threadfence();
-  const double* pb = partial + static_cast<int64_t>(b) * max_parts * D;
-  const double inv_T = 1.0 / static_cast<double>(T);
-  const int pairs = D >> 1;
-  double nn_all = 0.0;
-  for (int c0 = 0; c0 < pairs; c0 += kAnchorThreads) {   // uniform trip count: the per-head sums use block barriers
-    const int c = c0 + tid;
-    double t0 = 0.0, t1 = 0.0;
-    if (c < pairs) {
-      for (int p0 = 0; p0 < parts; p0 += 8) {
-        double2 v[8];
+  anchor_finish(b, parts, T, D, 1, partial, max_parts, tickets, m64, m32, mnorm2, ready, epoch);
+}
+
+// ------------------------------------------------------------------------------------------------
+// anchor pass, rows held in registers.  grid = one CTA per SM, kRowThreads threads.  The anchor rows of all chunks,
+// numbered chunk by chunk, are cut into equal runs, one per CTA.  A row is read by a SET of wpr consecutive warps
+// (wpr = 1 while a lane's share of the row is at most 48 columns); lane l of warp w of the set owns the 16-byte column
+// groups (w * 32 + l) + 32 * wpr * i, i < VPL.  The CTA's kRowWarps / wpr sets take the rows of the run round robin;
+// every lane
+//   converts its share of the row to fp64 once (the conversion unit's rate, a quarter of the fp64 multiply-add rate, is
+//   what bounds this kernel: one conversion per element, not one per phase) and issues the loads of its share of the
+//   set's next row into the registers just freed;
+//   phase 1: squares its share; the row's squared norm is a warp sum (plus an exchange between the set's warps through
+//            shared memory when wpr > 1); with per-head keys a sum over the 16 lanes that hold one head's 128 columns;
+//            1/|a| from the fp32 reciprocal square root and two Newton steps in fp64 (within a few units of the last
+//            place, the order of the rounding of the fp64 column sums themselves);
+//   phase 2: adds a / |a| to its own column sums, which stay in registers for the whole run.
+// Nothing is staged in shared memory and the sets never wait for one another inside the row loop.  At a chunk boundary
+// and at the end the sets' column sums are added in set order in shared memory, the CTA writes them as its slice of
+// that chunk and anchor_finish does the rest.
+// ------------------------------------------------------------------------------------------------
+constexpr int kRowThreads = 256;
+constexpr int kRowWarps = kRowThreads / 32;
+constexpr int kRowMaxVpl = 6;
+constexpr int kFusedMinCols = 2048;   // whole-token rows wider than this take the one-launch path (measured faster there)
+constexpr double kRowNorm2Hi = 1.2676506002282294e+30;    // 2^100: above it (or below 2^-80) 1/|a| is a true division
+
+__device__ __forceinline__ double rsqrt_newton(double x) {   // x in [2^-80, 2^100]: inside fp32's normal range
+  double y = static_cast<double>(rsqrtf(static_cast<float>(x)));
+  const double h = 0.5 * x;
+  y = fma(y, fma(-h * y, y, 0.5), y);
+  y = fma(y, fma(-h * y, y, 0.5), y);
+  return y;
+}
+__device__ __forceinline__ double inverse_norm(double n2) {
+  if (n2 >= kNorm2Lo && n2 <= kRowNorm2Hi) return rsqrt_newton(n2);
+  return n2 == 0.0 ? 0.0 : 1.0 / sqrt(n2);   // zero key: cosine 0; a NaN norm stays NaN
+}
+
+__device__ __forceinline__ void set_barrier(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// The lane's share of one row, converted to fp64 ONCE (x, kept in registers for phase 2), with the sum of squares of
+// each of its column groups.  One conversion instruction per element: the conversion unit's rate (a quarter of the
+// fp64 multiply-add rate) is what bounds the kernel, and converting once instead of once per phase is what the
+// registers are spent on.
+template <int VPL>
+__device__ __forceinline__ void row_convert(const uint4 (&q)[VPL], uint32_t active, double (&x)[8 * VPL], double (&p)[VPL]) {
 #pragma unroll
-        for (int pp = 0; pp < 8; ++pp)
-          v[pp] = p0 + pp < parts ? __ldcg(reinterpret_cast<const double2*>(pb + static_cast<int64_t>(p0 + pp) * D) + c)
-                                  : make_double2(0.0, 0.0);
+  for (int i = 0; i < VPL; ++i) {
+    const uint32_t w[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+    double* xi = x + 8 * i;
 #pragma unroll
-        for (int pp = 0; pp < 8; ++pp) {
-          t0 += v[pp].x;
-          t1 += v[pp].y;
-        }
-      }
-      t0 *= inv_T;
-      t1 *= inv_T;
-      reinterpret_cast<double2*>(m64 + static_cast<int64_t>(b) * D)[c] = make_double2(t0, t1);
-      reinterpret_cast<float2*>(m32 + static_cast<int64_t>(b) * D)[c] =
-          make_float2(static_cast<float>(t0), static_cast<float>(t1));
+    for (int e = 0; e < 4; ++e) {
+      xi[2 * e] = static_cast<double>(__uint_as_float(w[e] << 16));
+      xi[2 * e + 1] = static_cast<double>(__uint_as_float(w[e] & 0xFFFF0000u));
     }
-    const double nn = fma(t0, t0, t1 * t1);
-    if (hs == 1) {
-      nn_all += nn;
-    } else {
-      // 64 column pairs per head: warps 2j and 2j + 1 of this step hold head c0 / 64 + j
-      const double wsum = warp_sum(nn);
-      __syncthreads();
-      if (lane == 0) red[warp] = wsum;
-      __syncthreads();
-      const int head = (c0 >> 6) + tid;
-      if (tid < kAnchorWarps / 2 && head < hs)
-        mnorm2[(static_cast<int64_t>(b) * hs + head) * kMaxNormParts] = red[2 * tid] + red[2 * tid + 1];
-    }
-  }
-  if (hs == 1) {
-    const double wsum = warp_sum(nn_all);
-    if (lane == 0) red[warp] = wsum;
-    __syncthreads();
-    if (tid == 0) {
-      double t = 0.0;
-      for (int w = 0; w < kAnchorWarps; ++w) t += red[w];
-      mnorm2[static_cast<int64_t>(b) * kMaxNormParts] = t;
-    }
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    tickets[b] = 0;   // ready for the next call
-    if (ready) {
-      __threadfence();                                   // m64 / m32 / |m|^2 of every thread are out before the flag
-      *reinterpret_cast<volatile uint32_t*>(ready + b) = epoch;
-    }
+    double a = xi[0] * xi[0], c = xi[1] * xi[1];
+    a = fma(xi[2], xi[2], a); c = fma(xi[3], xi[3], c);
+    a = fma(xi[4], xi[4], a); c = fma(xi[5], xi[5], c);
+    a = fma(xi[6], xi[6], a); c = fma(xi[7], xi[7], c);
+    p[i] = (active >> i) & 1u ? a + c : 0.0;   // a column group past the end of the row repeats column 0: masked out
   }
 }
 
-template <int VPT>
-__global__ void __launch_bounds__(kAnchorThreads, VPT == 1 ? 4 : (VPT == 2 ? 3 : 2))
-anchor_pass(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int D, int hs, int G, int rpp,
-            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
-            float* __restrict__ m32, double* __restrict__ mnorm2, uint32_t* __restrict__ status) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(8) uint64_t bar[2];
-  dep_release();
-  if (threadIdx.x == 0) {
-    ptx::mbar_init(&bar[0], 1);
-    ptx::mbar_init(&bar[1], 1);
-    ptx::fence_mbar_init();
+// 1/|a| for each of the lane's column groups from their sums of squares (all equal with whole-token keys).
+template <int VPL>
+__device__ __forceinline__ void row_inverse_norms(const double (&p)[VPL], int hs, int wpr, int set, int wr, double* n2x,
+                                                  int& xc, double (&inv)[VPL]) {
+  const int lane = threadIdx.x & 31;
+  if (hs == 1) {
+    double n2 = p[0];
+#pragma unroll
+    for (int i = 1; i < VPL; ++i) n2 += p[i];
+    n2 = warp_sum(n2);
+    if (wpr > 1) {
+      // the set's warps leave their shares in one of two rows of n2x (alternating, so that one barrier per exchange
+      // is enough: a warp can only be one exchange ahead of the slowest warp of its set)
+      double* xs = n2x + (xc & 1) * kRowWarps + set * wpr;
+      ++xc;
+      if (lane == 0) xs[wr] = n2;
+      set_barrier(1 + set, wpr * 32);
+      if (wpr == 2) {
+        const double2 t = *reinterpret_cast<const double2*>(xs);
+        n2 = t.x + t.y;
+      } else if (wpr == 4) {
+        const double2 t = *reinterpret_cast<const double2*>(xs), u = *reinterpret_cast<const double2*>(xs + 2);
+        n2 = (t.x + t.y) + (u.x + u.y);
+      } else {
+        n2 = xs[0];
+        for (int w2 = 1; w2 < wpr; ++w2) n2 += xs[w2];
+      }
+    }
+    const double r = inverse_norm(n2);
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) inv[i] = r;
+  } else {
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) inv[i] = inverse_norm(half_warp_sum(p[i]));   // 16 lanes = 128 columns = one head
   }
-  __syncthreads();
-  uint32_t gbase = 0;
-  anchor_role<VPT>(smem, blockIdx.y, blockIdx.x, gridDim.x, K, stride, T, D, hs, G, rpp, partial, max_parts, tickets, m64,
-                   m32, mnorm2, status, nullptr, 0u, bar, gbase);
+}
+
+template <int VPL>
+__global__ void __launch_bounds__(kRowThreads, VPL <= 3 ? 2 : 1)
+anchor_rows(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, int T, int D, int hs, int wpr, int R,
+            double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
+            float* __restrict__ m32, double* __restrict__ mnorm2) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ __align__(16) double n2x[2 * kRowWarps];
+  double* sacc = reinterpret_cast<double*>(smem);   // [n_sets][D]
+  dep_release();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int n_sets = kRowWarps / wpr, set = warp / wpr, wr = warp - set * wpr;
+  const int vecs = D >> 3, vstep = 32 * wpr, v0 = wr * 32 + lane;
+  uint32_t active = 0;
+  int voff[VPL];
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) {
+    const bool on = v0 + i * vstep < vecs;
+    active |= (on ? 1u : 0u) << i;
+    voff[i] = on ? v0 + i * vstep : 0;
+  }
+  // the anchor rows of all chunks, numbered chunk by chunk, are cut into runs of R rows, one per CTA: every SM gets the
+  // same number of rows and a CTA hands in one slice per chunk its run touches (one or two at the benchmark shapes)
+  const int64_t total = static_cast<int64_t>(chunks) * T;
+  const int64_t g_end = min(total, static_cast<int64_t>(blockIdx.x + 1) * R);
+  int xc = 0;
+  for (int64_t g = static_cast<int64_t>(blockIdx.x) * R; g < g_end;) {
+    const int b = static_cast<int>(g / T);
+    const int r0 = static_cast<int>(g - static_cast<int64_t>(b) * T);
+    const int r1 = static_cast<int>(min(static_cast<int64_t>(T), r0 + (g_end - g)));
+    g += r1 - r0;
+    const uint4* Kb = reinterpret_cast<const uint4*>(K + static_cast<int64_t>(b) * stride);
+    // loads carry no predicate: a row past the end of the run is read from the chunk's last row and never used, and a
+    // column group past the end of the row is read from column 0 and masked out of the norm (its sums are not stored)
+    auto load_row = [&](int r, uint4 (&q)[VPL]) {
+      const uint4* row = Kb + static_cast<int64_t>(min(r, T - 1)) * vecs;
+#pragma unroll
+      for (int i = 0; i < VPL; ++i) q[i] = __ldcs(row + voff[i]);
+    };
+    double acc[8 * VPL];
+#pragma unroll
+    for (int i = 0; i < 8 * VPL; ++i) acc[i] = 0.0;
+    uint4 q[VPL];
+    int r = r0 + set;
+    load_row(r, q);
+    for (; r < r1; r += n_sets) {
+      double x[8 * VPL], p[VPL], inv[VPL];
+      row_convert<VPL>(q, active, x, p);
+      load_row(r + n_sets, q);   // the next row's loads fly while this one is finished
+      row_inverse_norms<VPL>(p, hs, wpr, set, wr, n2x, xc, inv);
+#pragma unroll
+      for (int i = 0; i < VPL; ++i)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[8 * i + e] = fma(x[8 * i + e], inv[i], acc[8 * i + e]);
+    }
+    // ---- every set leaves its column sums in its own row of sacc; the slice is their sum in set order
+    double* mine = sacc + static_cast<size_t>(set) * D;
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      if ((active >> i) & 1u) {
+        double2* dst = reinterpret_cast<double2*>(mine + 8 * voff[i]);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) dst[e] = make_double2(acc[8 * i + 2 * e], acc[8 * i + 2 * e + 1]);
+      }
+    }
+    __syncthreads();
+    // the CTAs whose runs touch chunk b, in order: first .. last; this one's slice number is its place among them
+    const int first = static_cast<int>((static_cast<int64_t>(b) * T) / R);
+    const int last = static_cast<int>((static_cast<int64_t>(b + 1) * T - 1) / R);
+    const int part = static_cast<int>(blockIdx.x) - first;
+    double2* my = reinterpret_cast<double2*>(partial + (static_cast<int64_t>(b) * max_parts + part) * D);
+    const int pairs = D >> 1;
+    for (int c = tid; c < pairs; c += kRowThreads) {
+      double2 t = reinterpret_cast<const double2*>(sacc)[c];
+      for (int s2 = 1; s2 < n_sets; ++s2) {
+        const double2 o = reinterpret_cast<const double2*>(sacc + static_cast<size_t>(s2) * D)[c];
+        t.x += o.x;
+        t.y += o.y;
+      }
+      __stcg(my + c, t);
+    }
+    anchor_finish(b, last - first + 1, T, D, hs, partial, max_parts, tickets, m64, m32, mnorm2, nullptr, 0u);
+    __syncthreads();   // sacc and anchor_finish's shared words are free for the next chunk
+  }
 }
 
 // Fallback for very wide rows (D > 8192): same arithmetic, accumulators in shared memory.
@@ -865,7 +1022,7 @@ compress_fused(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, 
     if (kind == -1) { ++idle; __nanosleep(200); continue; }
     if (kind == 0) {
       staged_chunk = -1;
-      anchor_role<VPT>(smem, item / parts, item % parts, parts, K, stride, T, D, 1, G, rpp, partial, max_parts, tickets_a,
+      anchor_role<VPT>(smem, item / parts, item % parts, parts, K, stride, T, D, G, rpp, partial, max_parts, tickets_a,
                        m64, m32, mnorm, status, ready, epoch, bar, gbase);
     } else if (kind == 1) {
       const int c = item / nblk;
@@ -945,14 +1102,14 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
 
 namespace {
 
-template <int VPT>
-void launch_anchor(dim3 grid, size_t smem, cudaStream_t s, const __nv_bfloat16* K, int64_t stride, int T, int D, int hs,
-                   int G, int rpp, double* partial, int max_parts, uint32_t* tickets, double* m64, float* m32,
-                   double* mnorm2, uint32_t* status) {
-  if (smem > 48 * 1024)
-    cudaFuncSetAttribute(anchor_pass<VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  anchor_pass<VPT><<<grid, kAnchorThreads, smem, s>>>(K, stride, T, D, hs, G, rpp, partial, max_parts, tickets, m64, m32,
-                                                      mnorm2, status);
+template <int VPL>
+void launch_rows(dim3 grid, size_t smem, cudaStream_t s, const __nv_bfloat16* K, int64_t stride, int chunks, int T, int D,
+                 int hs, int wpr, int R, double* partial, int max_parts, uint32_t* tickets, double* m64, float* m32,
+                 double* mnorm) {
+  if (smem > 40 * 1024)   // the kernel's static shared memory comes on top
+    cudaFuncSetAttribute(anchor_rows<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  anchor_rows<VPL><<<grid, kRowThreads, smem, s>>>(K, stride, chunks, T, D, hs, wpr, R, partial, max_parts, tickets, m64, m32,
+                                                   mnorm);
 }
 
 template <int VPT>
@@ -993,60 +1150,71 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
   if (smem_sel > 200 * 1024 || smem_m > 200 * 1024) return WK_ERR_SHAPE;
   wk_status st = WK_OK;
   if (need_scores) {
-    if (DF <= 8192) {
+    const bool select_here_f = !per_head && n_keep > 0 && n_keep < NA;
+    if (DF <= 8192 && select_here_f && DF > kFusedMinCols) {
+      // wide whole-token keys with a real selection: both passes in one launch (anchor CTAs and score CTAs side by side)
       // rows per group: two groups of G rows of DF bf16 in shared memory, at most one row per warp
       int G = kAnchorWarps;
       while (G > 1 && 2 * static_cast<size_t>(G) * DF * 2 > 100 * 1024) G >>= 1;
-      const int hs_a = per_head ? H : 1, nseg = kAnchorWarps / G;
-      const size_t smem_a = 2 * static_cast<size_t>(G) * DF * 2 +
-                            static_cast<size_t>(G) * (hs_a + (hs_a > nseg ? hs_a : nseg)) * sizeof(double);
-      // slices per chunk: as many CTAs as the machine holds at once, so that every SM carries the same number of them
-      // (a grid that leaves slots empty is spread unevenly: some SMs take their full share, others half of it)
-      int per_sm = static_cast<int>((220 * 1024) / (smem_a + 1024));
-      const int by_regs = DF > 2048 ? 2 : 4;
+      const int nseg = kAnchorWarps / G;
+      const size_t smem_a = 2 * static_cast<size_t>(G) * DF * 2 + static_cast<size_t>(G) * (1 + nseg) * sizeof(double);
+      const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 2 .. 4 here
+      const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
+      const size_t smem_s = smem_sel > smem_m ? smem_sel : smem_m;
+      const size_t smem_f = smem_a > smem_s ? smem_a : smem_s;
+      // persistent grid: what fits the machine at this shared-memory size
+      int per_sm = static_cast<int>((220 * 1024) / (smem_f + 2048));
+      const int by_regs = vpt == 1 ? 4 : (vpt == 2 ? 3 : 2);
       if (per_sm > by_regs) per_sm = by_regs;
-      // about a third more slices than CTA slots (measured: shorter items even out the end of the launch; flat between
-      // 1.2 and 1.6 slots' worth at both model shapes)
-      int parts = (ctx->sm_count * (per_sm < 1 ? 1 : per_sm) * 27 / 20 + chunks - 1) / chunks;
+      if (per_sm < 1) per_sm = 1;
+      // slices per chunk: about a third more than CTA slots (measured: shorter items even out the end of the launch;
+      // flat between 1.2 and 1.6 slots' worth)
+      int parts = (ctx->sm_count * per_sm * 27 / 20 + chunks - 1) / chunks;
       if (parts < 1) parts = 1;
       if (parts > max_parts) parts = max_parts;
       if (parts > (T + G - 1) / G) parts = (T + G - 1) / G;
       int rpp = (T + parts - 1) / parts;
       rpp = (rpp + G - 1) / G * G;            // whole groups, so that only a chunk's last slice has a short group
       parts = (T + rpp - 1) / rpp;
-      const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 1 .. 4 for DF <= 8192
-      if (!per_head && n_keep > 0 && n_keep < NA) {
-        // whole-key scoring with a real selection: both passes in one launch
-        const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
-        const size_t smem_s = smem_sel > smem_m ? smem_sel : smem_m;
-        const size_t smem_f = smem_a > smem_s ? smem_a : smem_s;
-        // persistent grid: what fits the machine at this shared-memory size (the same bound the slices were cut for)
-        int per_sm_f = static_cast<int>((220 * 1024) / (smem_f + 2048));
-        const int by_regs_f = vpt == 1 ? 4 : (vpt == 2 ? 3 : 2);
-        if (per_sm_f > by_regs_f) per_sm_f = by_regs_f;
-        if (per_sm_f < 1) per_sm_f = 1;
-        unsigned grid_f = static_cast<unsigned>(ctx->sm_count * per_sm_f);
-        const unsigned items = static_cast<unsigned>(chunks) * static_cast<unsigned>(parts + nblk);
-        if (grid_f > items) grid_f = items;
-        uint32_t* ready = tickets + 2 * ctx->max_batch;
-        FusedQueue* q = reinterpret_cast<FusedQueue*>(tickets + 3 * ctx->max_batch);
-        const uint32_t epoch = ++ctx->compress_epoch;
+      unsigned grid_f = static_cast<unsigned>(ctx->sm_count * per_sm);
+      const unsigned items = static_cast<unsigned>(chunks) * static_cast<unsigned>(parts + nblk);
+      if (grid_f > items) grid_f = items;
+      uint32_t* ready = tickets + 2 * ctx->max_batch;
+      FusedQueue* q = reinterpret_cast<FusedQueue*>(tickets + 3 * ctx->max_batch);
+      const uint32_t epoch = ++ctx->compress_epoch;
 #define WK_FUSED(V) launch_fused<V>(grid_f, smem_f, s, K, stride, chunks, T, NA, DF, n_keep, G, rpp, parts, nblk, ctx->sm_count, partial, max_parts, tickets, tickets + ctx->max_batch, ready, q, epoch, m64, m32, mnorm, s32, scores_out, keep_idx, ctx->status_dev)
-        if (vpt <= 1) WK_FUSED(1);
-        else if (vpt == 2) WK_FUSED(2);
-        else if (vpt == 3) WK_FUSED(3);
-        else WK_FUSED(4);
+      if (vpt <= 1) WK_FUSED(1);
+      else if (vpt == 2) WK_FUSED(2);
+      else if (vpt == 3) WK_FUSED(3);
+      else WK_FUSED(4);
 #undef WK_FUSED
-        return after_launch(ctx);
-      }
-      const dim3 grid(parts, chunks);
+      return after_launch(ctx);
+    } else if (DF <= 8192) {
+      // warps per row: the fewest that leave a lane at most kRowMaxVpl 16-byte column groups
+      const int vecs = DF / 8;
+      int wpr = 1;
+      while (wpr < kRowWarps && (vecs + 32 * wpr - 1) / (32 * wpr) > kRowMaxVpl) wpr <<= 1;
+      const int vpl = (vecs + 32 * wpr - 1) / (32 * wpr);
+      const int n_sets = kRowWarps / wpr;
       const int hs = per_head ? H : 1;
-#define WK_ANCHOR(V) launch_anchor<V>(grid, smem_a, s, K, stride, T, DF, hs, G, rpp, partial, max_parts, tickets, m64, m32, mnorm, ctx->status_dev)
-      if (vpt <= 1) WK_ANCHOR(1);
-      else if (vpt == 2) WK_ANCHOR(2);
-      else if (vpt == 3) WK_ANCHOR(3);
-      else WK_ANCHOR(4);
-#undef WK_ANCHOR
+      const size_t smem_r = static_cast<size_t>(n_sets) * DF * sizeof(double);
+      // rows per CTA: an even share of all chunks' anchor rows, and never so few that a chunk is cut into more slices
+      // than the scratch holds
+      const int64_t total = static_cast<int64_t>(chunks) * T;
+      int64_t R = (total + ctx->sm_count - 1) / ctx->sm_count;
+      const int64_t r_min = (T + max_parts - 2) / (max_parts - 1);
+      if (R < r_min) R = r_min;
+      const dim3 grid(static_cast<unsigned>((total + R - 1) / R));
+#define WK_ROWS(V) launch_rows<V>(grid, smem_r, s, K, stride, chunks, T, DF, hs, wpr, static_cast<int>(R), partial, max_parts, tickets, m64, m32, mnorm)
+      switch (vpl) {
+        case 1: WK_ROWS(1); break;
+        case 2: WK_ROWS(2); break;
+        case 3: WK_ROWS(3); break;
+        case 4: WK_ROWS(4); break;
+        case 5: WK_ROWS(5); break;
+        default: WK_ROWS(6); break;
+      }
+#undef WK_ROWS
     } else {
       if (per_head) return WK_ERR_SHAPE;   // rows wider than 8,192 columns take the whole-key fallback only
       const dim3 grid_a(max_parts, chunks);
