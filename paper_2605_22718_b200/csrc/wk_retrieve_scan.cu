@@ -40,6 +40,7 @@ constexpr int kScanMaxBlocks = 1024;
 
 constexpr int kSampleBlocks = 128;          // scan_sample's grid
 constexpr int kSampleThreads = 256;
+constexpr int kSampleBatch = 4;             // samples a thread has in flight
 constexpr uint32_t kSurvivorCap = 1u << 20;  // entries of the survivor list
 
 struct ScanHeader {
@@ -112,45 +113,60 @@ scan_sample(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   // sample s is candidate floor(s * n / n_samples) (integer arithmetic); block b takes samples b, b + gridDim.x, ...; class of a sample =
   // its position in the block's sequence modulo k, so that classes are disjoint sets of candidates
   const int64_t per_block = (n_samples + gridDim.x - 1) / gridDim.x;
-  // the weight pi / (largest t) of the key comes from the block's first 256 samples (any positive weight gives valid
-  // pivots, a rough one just picks slightly different ones); the record's t_max covers all of the block's samples
-  float tmax = 0.f;
-  {
-    const int64_t smp = static_cast<int64_t>(tid) * gridDim.x + blockIdx.x;
-    if (tid < per_block && smp < n_samples) {
-      const int64_t i = smp * n / n_samples;
-      if (!(valid && !__ldg(valid + i))) {
-        float t32, adot32;
-        cheap_terms(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v, t32, adot32);
-        if (t32 < 3.0e38f && adot32 < 3.0e38f) tmax = t32;   // false for NaN and Inf: not a candidate
+  // A thread takes positions tid, tid + 256, ... of the block's sequence, kSampleBatch at a time: the loads of a batch
+  // are all issued before the first is used, so that a batch is one trip to memory instead of four in a row.  (What is
+  // left is the rate at which DRAM opens rows: every sample is a 32-byte read from a row of its own.)
+  // The weight pi / (largest t) of the key comes from the block's first 256 samples (any positive weight gives valid
+  // pivots, a rough one just picks slightly different ones); the record's t_max covers all of the block's samples.
+  float tmax = 0.f, dmin = 2.f, wt = 0.f;
+  for (int64_t q0 = 0; q0 < per_block; q0 += kSampleBatch * kSampleThreads) {   // the same trips for every thread
+    float4 a[kSampleBatch], b[kSampleBatch];
+    int64_t ci[kSampleBatch];
+    int vflag[kSampleBatch];
+    bool ok[kSampleBatch];
+#pragma unroll
+    for (int u = 0; u < kSampleBatch; ++u) {
+      const int64_t q = q0 + u * kSampleThreads + tid;
+      const int64_t smp = q * gridDim.x + blockIdx.x;
+      ok[u] = q < per_block && smp < n_samples;
+      ci[u] = ok[u] ? smp * n / n_samples : 0;   // n_samples <= n: strictly increasing in smp, so samples are distinct
+      vflag[u] = 1;
+      a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      b[u] = a[u];
+      if (ok[u]) {
+        if (valid) vflag[u] = __ldg(valid + ci[u]);
+        a[u] = __ldg(poses + 2 * ci[u]);
+        b[u] = __ldg(poses + 2 * ci[u] + 1);
       }
     }
-  }
+    float t32[kSampleBatch], ad32[kSampleBatch];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-  if (lane == 0) s_tmax[warp] = tmax;
-  __syncthreads();
-  float est = s_tmax[0];
-  for (int w = 1; w < kSampleThreads / 32; ++w) est = fmaxf(est, s_tmax[w]);
-  __syncthreads();
-  const float wt = est > 0.f ? 3.14159274f / est : 0.f;
-  tmax = 0.f;
-  float dmin = 2.f;
-  for (int64_t q = tid; q < per_block; q += kSampleThreads) {
-    const int64_t smp = q * gridDim.x + blockIdx.x;
-    if (smp >= n_samples) break;
-    const int64_t i = smp * n / n_samples;   // n_samples <= n: strictly increasing in smp, so samples are distinct
-    if (valid && !__ldg(valid + i)) continue;
-    float t32, adot32;
-    cheap_terms(__ldg(poses + 2 * i), __ldg(poses + 2 * i + 1), cur.v, t32, adot32);
-    if (!(t32 < 3.0e38f && adot32 < 3.0e38f)) continue;
-    tmax = fmaxf(tmax, t32);
-    dmin = fminf(dmin, adot32);
-    if (k > 0) {
-      const float om = fmaxf(0.f, 1.f - adot32);
-      const float key = 2.f * sqrtf(om + om) + wt * t32;   // ~ r + pi t / max t, non-negative
-      atomicMin(&s_best[static_cast<int>(q % k)],
-                (static_cast<unsigned long long>(__float_as_uint(key)) << 32) | static_cast<unsigned long long>(i));
+    for (int u = 0; u < kSampleBatch; ++u) {
+      cheap_terms(a[u], b[u], cur.v, t32[u], ad32[u]);
+      ok[u] = ok[u] && vflag[u] != 0 && t32[u] < 3.0e38f && ad32[u] < 3.0e38f;   // false for NaN and Inf: not a candidate
+    }
+    if (q0 == 0) {
+      float est = ok[0] ? t32[0] : 0.f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) est = fmaxf(est, __shfl_xor_sync(0xffffffffu, est, o));
+      if (lane == 0) s_tmax[warp] = est;
+      __syncthreads();
+      est = s_tmax[0];
+      for (int w = 1; w < kSampleThreads / 32; ++w) est = fmaxf(est, s_tmax[w]);
+      __syncthreads();
+      wt = est > 0.f ? 3.14159274f / est : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < kSampleBatch; ++u) {
+      if (!ok[u]) continue;
+      tmax = fmaxf(tmax, t32[u]);
+      dmin = fminf(dmin, ad32[u]);
+      if (k > 0) {
+        const float om = fmaxf(0.f, 1.f - ad32[u]);
+        const float key = 2.f * sqrtf(om + om) + wt * t32[u];   // ~ r + pi t / max t, non-negative
+        atomicMin(&s_best[static_cast<int>((q0 + u * kSampleThreads + tid) % k)],
+                  (static_cast<unsigned long long>(__float_as_uint(key)) << 32) | static_cast<unsigned long long>(ci[u]));
+      }
     }
   }
 #pragma unroll
@@ -315,7 +331,26 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
       }
     }
   }
-  if (wcnt > 0) flush();
+  {
+    // what is left in the warps' buffers at the end: one atomic for the whole block (every warp of every block arrives
+    // here at about the same time, and thousands of atomics on one word would queue up)
+    __shared__ int s_wcnt[kScanThreads / 32];
+    __shared__ uint32_t s_base;
+    if (lane == 0) s_wcnt[warp] = wcnt;
+    __syncthreads();
+    if (tid == 0) {
+      int total = 0;
+      for (int w = 0; w < kScanThreads / 32; ++w) total += s_wcnt[w];
+      s_base = total > 0 ? atomicAdd(&h->n_surv, static_cast<uint32_t>(total)) : 0u;
+    }
+    __syncthreads();
+    uint32_t base = s_base;
+    for (int w = 0; w < warp; ++w) base += static_cast<uint32_t>(s_wcnt[w]);
+    for (int j = lane; j < wcnt; j += 32) {
+      if (base + j < kSurvivorCap) surv[base + j] = wbuf[j];
+      else h->overflow = 1u;
+    }
+  }
   if (bad) atomicOr(status, WK_DEV_NONFINITE);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -331,17 +366,42 @@ scan_filter(const float4* __restrict__ poses, const int32_t* __restrict__ valid,
   }
 }
 
+// Rank of each of n entries under (key, index), by counting, with all of the block's threads: P threads share an entry
+// (each counts over every P-th other entry), P the largest power of two with n * P <= blockDim.x.  rank[] is shared
+// memory of at least n words.  Ends with a block barrier.
+__device__ __forceinline__ void block_rank(const unsigned long long* key, const int32_t* idx, int n, int* rank) {
+  for (int e = threadIdx.x; e < n; e += blockDim.x) rank[e] = 0;
+  __syncthreads();
+  int shift = 0;
+  while (shift < 5 && (n << (shift + 1)) <= static_cast<int>(blockDim.x)) ++shift;
+  const int P = 1 << shift;
+  for (int slot = threadIdx.x; slot < (n << shift); slot += blockDim.x) {
+    const int e = slot >> shift, p = slot & (P - 1);
+    const unsigned long long ke = key[e];
+    const int32_t ie = idx[e];
+    int r = 0;
+#pragma unroll 4
+    for (int u = p; u < n; u += P) {
+      const unsigned long long ku = key[u];
+      r += (ku < ke) || (ku == ke && idx[u] < ie);
+    }
+    if (r) atomicAdd(&rank[e], r);
+  }
+  __syncthreads();
+}
+
 // The k best (distance, index) pairs seen so far by one block, in shared memory.  Distances are non-negative, so their
 // bit patterns order like the values and every comparison is an integer one.
 struct TopK {
   unsigned long long* key;   // [2][kScanCap] distance bits
   int32_t* idx;              // [2][kScanCap]
+  int* rank_s;               // [kScanCap] scratch of compact()
   int* cnt;                  // entries in the list
   double* tau;               // current k-th best distance (+inf until k entries are known)
   int k;
 
-  __device__ __forceinline__ void init(unsigned long long* k_, int32_t* i_, int* c_, double* t_, int kk) {
-    key = k_; idx = i_; cnt = c_; tau = t_; k = kk;
+  __device__ __forceinline__ void init(unsigned long long* k_, int32_t* i_, int* r_, int* c_, double* t_, int kk) {
+    key = k_; idx = i_; rank_s = r_; cnt = c_; tau = t_; k = kk;
     if (threadIdx.x == 0) { *cnt = 0; *tau = INFINITY; }
     __syncthreads();
   }
@@ -358,27 +418,55 @@ struct TopK {
   // Cuts the list back to its k best, sorted, by exact rank counting (quadratic in the list length, which is why the
   // list is kept short); all threads of the block call it together.
   __device__ __forceinline__ void compact() {
+    __shared__ unsigned long long s_gmin[kScanMaxK];
+    __shared__ unsigned long long s_cut;
+    __shared__ int s_m;
     __syncthreads();
     const int n = *cnt;
     unsigned long long* key2 = key + kScanCap;
     int32_t* i2 = idx + kScanCap;
+    // Counting ranks costs n^2 comparisons, so a long list is thinned first: deal the entries into k groups; the
+    // largest of the groups' minima has k entries at or below it, so nothing above it is among the k best.
+    const bool thin = k > 0 && n > 4 * k;
+    if (threadIdx.x < kScanMaxK) s_gmin[threadIdx.x] = ~0ull;
+    if (threadIdx.x == 0) { s_m = 0; s_cut = ~0ull; }
+    __syncthreads();
+    if (thin) {
+      for (int e = threadIdx.x; e < n; e += blockDim.x) atomicMin(&s_gmin[e % k], key[e]);
+      __syncthreads();
+      if (threadIdx.x < 32) {
+        unsigned long long v = 0ull;
+        for (int g = threadIdx.x; g < k; g += 32) v = s_gmin[g] > v ? s_gmin[g] : v;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
+          v = w > v ? w : v;
+        }
+        if (threadIdx.x == 0) s_cut = v;
+      }
+      __syncthreads();
+    }
+    const unsigned long long cut = s_cut;
     for (int e = threadIdx.x; e < n; e += blockDim.x) {
       const unsigned long long ke = key[e];
-      const int32_t ie = idx[e];
-      int rank = 0;
-#pragma unroll 4
-      for (int u = 0; u < n; ++u) {
-        const unsigned long long ku = key[u];
-        rank += (ku < ke) || (ku == ke && idx[u] < ie);
+      if (ke <= cut) {
+        const int pos = atomicAdd(&s_m, 1);
+        key2[pos] = ke;
+        i2[pos] = idx[e];
       }
-      if (rank < k) { key2[rank] = ke; i2[rank] = ie; }
     }
     __syncthreads();
-    const int m = n < k ? n : k;
-    for (int e = threadIdx.x; e < m; e += blockDim.x) { key[e] = key2[e]; idx[e] = i2[e]; }
+    const int n2 = s_m;
+    block_rank(key2, i2, n2, rank_s);
+    for (int e = threadIdx.x; e < n2; e += blockDim.x) {
+      const int rank = rank_s[e];
+      if (rank < k) { key[rank] = key2[e]; idx[rank] = i2[e]; }
+    }
+    const int m = n2 < k ? n2 : k;
+    __syncthreads();
     if (threadIdx.x == 0) {
       *cnt = m;
-      *tau = (m == k && k > 0) ? __longlong_as_double(static_cast<long long>(key2[k - 1])) : INFINITY;
+      *tau = (m == k && k > 0) ? __longlong_as_double(static_cast<long long>(key[k - 1])) : INFINITY;
     }
     __syncthreads();
   }
@@ -392,6 +480,7 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
             double* __restrict__ dist_out) {
   __shared__ unsigned long long s_key[2 * kScanCap];
   __shared__ int32_t s_i[2 * kScanCap];
+  __shared__ int s_rank[2 * kScanCap];
   __shared__ __align__(8) int32_t s_pend[kPendLow + kScanUnroll * kSelThreads];   // candidates that passed the cheap bound
   __shared__ int s_cnt, s_npend[2];
   __shared__ uint32_t s_last;
@@ -401,7 +490,7 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
   dep_wait();
   dep_release();
   TopK top;
-  top.init(s_key, s_i, &s_cnt, &s_tau, k);
+  top.init(s_key, s_i, s_rank, &s_cnt, &s_tau, k);
   // what is walked: the survivor list, or -- if it overflowed -- every pose (entry e is then candidate e)
   const bool listed = h->overflow == 0u;
   const int64_t n = listed ? static_cast<int64_t>(h->n_surv) : n_all;
@@ -452,15 +541,17 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
   // only lengthen a short kernel)
   const int64_t warm0 = static_cast<int64_t>(blockIdx.x) * kScanWarm;
   const int64_t warm_all = listed ? 0 : static_cast<int64_t>(gridDim.x) * kScanWarm;
-  if (k > 0 && !listed && threadIdx.x < kScanWarm) {
-    const int64_t e = warm0 + threadIdx.x;
-    if (e < n) {
-      const int32_t i = cand_of(e);
-      if (!(valid && !__ldg(valid + i))) exact(i, INFINITY);
+  if (!listed) {
+    if (k > 0 && threadIdx.x < kScanWarm) {
+      const int64_t e = warm0 + threadIdx.x;
+      if (e < n) {
+        const int32_t i = cand_of(e);
+        if (!(valid && !__ldg(valid + i))) exact(i, INFINITY);
+      }
     }
+    top.compact();
+    refresh();
   }
-  top.compact();
-  refresh();
   const int64_t step = static_cast<int64_t>(gridDim.x) * kSelThreads;
   const int64_t lane_off = warm_all + static_cast<int64_t>(blockIdx.x) * kSelThreads + threadIdx.x;
   const int64_t rest = n > warm_all ? n - warm_all : 0;
@@ -517,7 +608,7 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
     if (__syncthreads_or(*reinterpret_cast<volatile int*>(&s_npend[0]) > kPendLow)) drain();
   }
   __syncthreads();
-  drain();
+  if (!listed) drain();
   top.compact();
   for (int e = threadIdx.x; e < k; e += blockDim.x) {
     ScanEntry o;
@@ -565,11 +656,13 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
     heads[l] = f.i >= 0 ? static_cast<unsigned long long>(__double_as_longlong(f.d)) : kInf;
   }
   __syncthreads();
-  if (n_lists >= k) {
-    for (int l = tid; l < n_lists; l += blockDim.x) {
+  // (any k lists give a valid cut; the first 128 keep the counting short and still leave only a few k entries)
+  const int n_heads = n_lists < 128 ? n_lists : 128;
+  if (n_heads >= k) {
+    for (int l = tid; l < n_heads; l += blockDim.x) {
       const unsigned long long hl = heads[l];
       int rank = 0;
-      for (int u = 0; u < n_lists; ++u) {
+      for (int u = 0; u < n_heads; ++u) {
         const unsigned long long hu = heads[u];
         rank += (hu < hl) || (hu == hl && u < l);
       }
@@ -593,17 +686,12 @@ scan_select(const float4* __restrict__ poses, const int32_t* __restrict__ valid_
   const int n_g = s_cnt;
   if (n_g <= kGather) {
     // exact rank under (distance, index) among the gathered entries
+    block_rank(s_key, s_i, n_g, s_rank);
     for (int e = tid; e < n_g; e += blockDim.x) {
-      const unsigned long long ke = s_key[e];
-      const int32_t ie = s_i[e];
-      int rank = 0;
-      for (int u = 0; u < n_g; ++u) {
-        const unsigned long long ku = s_key[u];
-        rank += (ku < ke) || (ku == ke && s_i[u] < ie);
-      }
+      const int rank = s_rank[e];
       if (rank < k && rank < out_capacity) {
-        ids_out[rank] = ie;
-        if (dist_out) dist_out[rank] = __longlong_as_double(static_cast<long long>(ke));
+        ids_out[rank] = s_i[e];
+        if (dist_out) dist_out[rank] = __longlong_as_double(static_cast<long long>(s_key[e]));
       }
     }
     return;
