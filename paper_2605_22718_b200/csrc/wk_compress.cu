@@ -30,7 +30,7 @@ namespace {
 
 constexpr int kMaxNormParts = 32;     // pitch of the per-problem |m|^2 record in scratch (one share is used)
 constexpr int kScoreThreads = 256;
-constexpr int kScoreRowsPerCta = 32;
+constexpr int kScoreRowsPerCta = 32;   // head_score's block of rows; score_select / compress_fused get theirs at launch
 
 __device__ __forceinline__ double bf16_to_f64(uint32_t bits16) {
   return static_cast<double>(__uint_as_float(bits16 << 16));
@@ -395,6 +395,7 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
 constexpr int kRowMaxVpl = 6;
+constexpr int kFusedScoreRows = 64;   // rows of a score item of the one-launch kernel (measured: 64-80 best at 5,120 columns)
 constexpr int kFusedMinCols = 2048;   // whole-token rows wider than this take the one-launch path (measured faster there)
 constexpr double kRowNorm2Hi = 1.2676506002282294e+30;    // 2^100: above it (or below 2^-80) 1/|a| is a true division
 
@@ -830,7 +831,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
 }
 
 // ------------------------------------------------------------------------------------------------
-// score pass + selection.  grid = blocks of kScoreRowsPerCta rows, problem-major (blockIdx.x = b * nblk + block), so that
+// score pass + selection.  grid = blocks of rows (nblk equal blocks per chunk, sized at launch), problem-major (blockIdx.x = b * nblk + block), so that
 // the problems finish in order; one warp per row; m32 staged in shared memory.  The CTA that hands in the last rows of
 // a problem (atomic ticket; nobody waits) runs that problem's selection on the spot, under the streaming of the
 // problems behind it.
@@ -838,7 +839,7 @@ select_pass(const __nv_bfloat16* __restrict__ K, RowMap rm, int T, int NA, int D
 // the packed pairs), one addition of the two, then five shuffle additions: no deeper than the single chain of
 // 8 * ceil(D/256) + 5 operations the selection's error band is derived for.
 // ------------------------------------------------------------------------------------------------
-// The work of one score CTA: block `blk` (kScoreRowsPerCta rows) of chunk b, and the chunk's selection if this CTA hands in
+// The work of one score CTA: block `blk` (one of nblk equal blocks of rows) of chunk b, and the chunk's selection if this CTA hands in
 // the chunk's last block.
 __device__ __forceinline__ bool score_role(uint8_t* smem, int b, int blk, const __nv_bfloat16* __restrict__ K, int64_t stride,
                                            int T, int NA, int D, int n_keep, int nblk, const float* __restrict__ m32,
@@ -857,8 +858,9 @@ __device__ __forceinline__ bool score_role(uint8_t* smem, int b, int blk, const 
     __syncthreads();
   }
   const int vecs = D >> 3;
-  const int j0 = blk * kScoreRowsPerCta;
-  const int j1 = min(NA, j0 + kScoreRowsPerCta);
+  const int rows = (NA + nblk - 1) / nblk;   // the chunk's non-anchor rows in nblk equal blocks
+  const int j0 = min(NA, blk * rows);
+  const int j1 = min(NA, j0 + rows);
   const int pitch = D;
   const __nv_bfloat16* Kb = K + static_cast<int64_t>(b) * stride + static_cast<int64_t>(T) * pitch;
   // two rows per warp at a time, so that twice as many 16-byte loads are in flight
@@ -1159,7 +1161,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       const int nseg = kAnchorWarps / G;
       const size_t smem_a = 2 * static_cast<size_t>(G) * DF * 2 + static_cast<size_t>(G) * (1 + nseg) * sizeof(double);
       const int vpt = (DF / 8 + kAnchorThreads - 1) / kAnchorThreads;   // 2 .. 4 here
-      const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
+      const int nblk = (NA + kFusedScoreRows - 1) / kFusedScoreRows;
       const size_t smem_s = smem_sel > smem_m ? smem_sel : smem_m;
       const size_t smem_f = smem_a > smem_s ? smem_a : smem_s;
       // persistent grid: what fits the machine at this shared-memory size
@@ -1226,7 +1228,16 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
                                                                 mnorm);
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
-    const int nblk = (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta;
+    // score_select's blocks of rows: whole rounds of its 8 warps x 2 rows, and as few full waves of CTAs (four resident
+    // per SM) as blocks of at most 128 rows allow -- a last wave that is nearly empty costs as much as a full one
+    int srows = 128;
+    for (int waves = 1; waves <= 64; ++waves) {
+      const int64_t per = (static_cast<int64_t>(NA) * chunks + static_cast<int64_t>(ctx->sm_count) * 4 * waves - 1) /
+                          (static_cast<int64_t>(ctx->sm_count) * 4 * waves);
+      const int r16 = static_cast<int>((per + 15) / 16 * 16);
+      if (r16 <= 128) { srows = r16 < 16 ? 16 : r16; break; }
+    }
+    const int nblk = per_head ? (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta : (NA + srows - 1) / srows;
     if (per_head) {
       if (smem_m > 48 * 1024)
         WK_CUDA_TRY(ctx, cudaFuncSetAttribute(head_score, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_m)));
