@@ -38,6 +38,9 @@ def test_device_generators_match_numpy():
     (100, 3, 50, 2, 0.05),
     (256, 12, 128, 2, 0.1),       # Matrix-Game row width
     (64, 40, 32, 1, 0.05),        # LingBot row width
+    (200, 16, 100, 3, 0.1),       # 2,048 columns: two warps share a row of the anchor pass
+    (96, 13, 48, 2, 0.1),         # 1,664 columns: two warps per row, some lanes without a column group
+    (45, 20, 30, 5, 0.1),         # wide rows, several short chunks
 ])
 def test_compress_matches_oracle(T, H, n_keep, batch, sigma):
     D = H * 128
@@ -77,6 +80,31 @@ def test_compress_retention_ladder_and_degenerate_inputs():
     keep = kv.compress_chunk(wd.to_device_bf16(Kz)[None]).cpu().numpy()[0]
     np.testing.assert_array_equal(keep, o.compress_chunk(Kz, T, T // 2)[0])
     assert kv.poll_status() == (0, 0)
+
+
+@pytest.mark.parametrize("H", [2, 12, 40])
+def test_compress_scores_only_and_extreme_row_norms(H):
+    """Keep everything but ask for the scores (the anchor pass and the score pass run, no selection), on keys whose
+    anchor rows span 2^-70 .. 2^70 in scale: cosine scores do not depend on a row's scale, and 1/|a| leaves the range of
+    the fast reciprocal square root for the true division."""
+    T = 40
+    D = H * 128
+    bits = wi.key_chunk_bf16(5, 1, 3, T, D, 0.1)
+    scale = np.ones(3 * T, dtype=np.float32)
+    scale[0], scale[1], scale[2], scale[3] = 2.0 ** 70, 2.0 ** -70, 2.0 ** 55, 2.0 ** -45
+    scale[T + 1], scale[T + 2] = 2.0 ** 40, 2.0 ** -40
+    f32 = (bits.astype(np.uint32) << 16).view(np.float32) * scale[:, None]   # a power of two keeps the 8-bit mantissa
+    Kb = (f32.view(np.uint32) >> 16).astype(np.uint16)
+    assert np.array_equal((Kb.astype(np.uint32) << 16).view(np.float32), f32)
+    kv = make_kv(n_layers=1, n_heads=H, tokens_per_frame=T, n_keep=2 * T, pool_slots=1, max_k=1)
+    scores = torch.empty((1, 2 * T), dtype=torch.float32, device="cuda")
+    keep = kv.compress_chunk(wd.to_device_bf16(Kb)[None], scores_out=scores).cpu().numpy()[0]
+    np.testing.assert_array_equal(keep, np.arange(3 * T))
+    assert kv.poll_status() == (0, 0)
+    np.testing.assert_allclose(scores[0].cpu().numpy(), o.compression_scores_definitional(Kb, T), atol=2e-6)
+    # the same keys unscaled give the same scores: the scale of a row cancels in a cosine
+    np.testing.assert_allclose(o.compression_scores_definitional(Kb, T), o.compression_scores_definitional(bits, T),
+                               atol=1e-12)
 
 
 # ----------------------------------------------------------------------------- pool + retrieval
