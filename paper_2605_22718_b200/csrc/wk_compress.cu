@@ -375,10 +375,10 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
 }
 
 // ------------------------------------------------------------------------------------------------
-// anchor pass, rows held in registers.  grid = one CTA per SM, kRowThreads threads.  The anchor rows of all chunks,
+// anchor pass, rows held in registers.  grid = one CTA per SM, NW warps.  The anchor rows of all chunks,
 // numbered chunk by chunk, are cut into equal runs, one per CTA.  A row is read by a SET of wpr consecutive warps
-// (wpr = 1 while a lane's share of the row is at most 48 columns); lane l of warp w of the set owns the 16-byte column
-// groups (w * 32 + l) + 32 * wpr * i, i < VPL.  The CTA's kRowWarps / wpr sets take the rows of the run round robin;
+// (the fewest that leave a lane at most 6, with per-head keys 3, 16-byte column groups); lane l of warp w of the set owns the column
+// groups (w * 32 + l) + 32 * wpr * i, i < VPL.  The CTA's NW / wpr sets take the rows of the run round robin;
 // every lane
 //   converts its share of the row to fp64 once (the conversion unit's rate, a quarter of the fp64 multiply-add rate, is
 //   what bounds this kernel: one conversion per element, not one per phase) and issues the loads of its share of the
@@ -392,9 +392,11 @@ __device__ __forceinline__ void anchor_role(uint8_t* smem, int b, int part, int 
 // and at the end the sets' column sums are added in set order in shared memory, the CTA writes them as its slice of
 // that chunk and anchor_finish does the rest.
 // ------------------------------------------------------------------------------------------------
-constexpr int kRowThreads = 256;
-constexpr int kRowWarps = kRowThreads / 32;
-constexpr int kRowMaxVpl = 6;
+// NW warps per CTA and at most kRowMaxVpl column groups per lane: 8 warps x 6 groups for whole-token keys (255 registers
+// per thread), 16 warps x 3 groups for per-head keys (128 registers; measured faster there: 109 against 124 us per cfg2
+// call, 624 against 690 us at the LingBot shape -- and 2 us slower for whole-token keys).
+constexpr int kRowWarpsWhole = 8, kRowMaxVplWhole = 6;
+constexpr int kRowWarpsHead = 16, kRowMaxVplHead = 3;
 constexpr int kFusedScoreRows = 64;   // rows of a score item of the one-launch kernel (measured: 64-80 best at 5,120 columns)
 constexpr int kFusedMinCols = 2048;   // whole-token rows wider than this take the one-launch path (measured faster there)
 constexpr double kRowNorm2Hi = 1.2676506002282294e+30;    // 2^100: above it (or below 2^-80) 1/|a| is a true division
@@ -439,7 +441,7 @@ __device__ __forceinline__ void row_convert(const uint4 (&q)[VPL], uint32_t acti
 }
 
 // 1/|a| for each of the lane's column groups from their sums of squares (all equal with whole-token keys).
-template <int VPL>
+template <int VPL, int NW>
 __device__ __forceinline__ void row_inverse_norms(const double (&p)[VPL], int hs, int wpr, int set, int wr, double* n2x,
                                                   int& xc, double (&inv)[VPL]) {
   const int lane = threadIdx.x & 31;
@@ -451,7 +453,7 @@ __device__ __forceinline__ void row_inverse_norms(const double (&p)[VPL], int hs
     if (wpr > 1) {
       // the set's warps leave their shares in one of two rows of n2x (alternating, so that one barrier per exchange
       // is enough: a warp can only be one exchange ahead of the slowest warp of its set)
-      double* xs = n2x + (xc & 1) * kRowWarps + set * wpr;
+      double* xs = n2x + (xc & 1) * NW + set * wpr;
       ++xc;
       if (lane == 0) xs[wr] = n2;
       set_barrier(1 + set, wpr * 32);
@@ -475,17 +477,17 @@ __device__ __forceinline__ void row_inverse_norms(const double (&p)[VPL], int hs
   }
 }
 
-template <int VPL>
-__global__ void __launch_bounds__(kRowThreads, VPL <= 3 ? 2 : 1)
+template <int VPL, int NW>
+__global__ void __launch_bounds__(NW * 32, 1)
 anchor_rows(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, int T, int D, int hs, int wpr, int R,
             double* __restrict__ partial, int max_parts, uint32_t* __restrict__ tickets, double* __restrict__ m64,
             float* __restrict__ m32, double* __restrict__ mnorm2) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ __align__(16) double n2x[2 * kRowWarps];
+  __shared__ __align__(16) double n2x[2 * NW];
   double* sacc = reinterpret_cast<double*>(smem);   // [n_sets][D]
   dep_release();
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int n_sets = kRowWarps / wpr, set = warp / wpr, wr = warp - set * wpr;
+  const int n_sets = NW / wpr, set = warp / wpr, wr = warp - set * wpr;
   const int vecs = D >> 3, vstep = 32 * wpr, v0 = wr * 32 + lane;
   uint32_t active = 0;
   int voff[VPL];
@@ -523,7 +525,7 @@ anchor_rows(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, int
       double x[8 * VPL], p[VPL], inv[VPL];
       row_convert<VPL>(q, active, x, p);
       load_row(r + n_sets, q);   // the next row's loads fly while this one is finished
-      row_inverse_norms<VPL>(p, hs, wpr, set, wr, n2x, xc, inv);
+      row_inverse_norms<VPL, NW>(p, hs, wpr, set, wr, n2x, xc, inv);
 #pragma unroll
       for (int i = 0; i < VPL; ++i)
 #pragma unroll
@@ -546,7 +548,7 @@ anchor_rows(const __nv_bfloat16* __restrict__ K, int64_t stride, int chunks, int
     const int part = static_cast<int>(blockIdx.x) - first;
     double2* my = reinterpret_cast<double2*>(partial + (static_cast<int64_t>(b) * max_parts + part) * D);
     const int pairs = D >> 1;
-    for (int c = tid; c < pairs; c += kRowThreads) {
+    for (int c = tid; c < pairs; c += NW * 32) {
       double2 t = reinterpret_cast<const double2*>(sacc)[c];
       for (int s2 = 1; s2 < n_sets; ++s2) {
         const double2 o = reinterpret_cast<const double2*>(sacc + static_cast<size_t>(s2) * D)[c];
@@ -1104,13 +1106,13 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
 
 namespace {
 
-template <int VPL>
+template <int VPL, int NW>
 void launch_rows(dim3 grid, size_t smem, cudaStream_t s, const __nv_bfloat16* K, int64_t stride, int chunks, int T, int D,
                  int hs, int wpr, int R, double* partial, int max_parts, uint32_t* tickets, double* m64, float* m32,
                  double* mnorm) {
   if (smem > 40 * 1024)   // the kernel's static shared memory comes on top
-    cudaFuncSetAttribute(anchor_rows<VPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
-  anchor_rows<VPL><<<grid, kRowThreads, smem, s>>>(K, stride, chunks, T, D, hs, wpr, R, partial, max_parts, tickets, m64, m32,
+    cudaFuncSetAttribute(anchor_rows<VPL, NW>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  anchor_rows<VPL, NW><<<grid, NW * 32, smem, s>>>(K, stride, chunks, T, D, hs, wpr, R, partial, max_parts, tickets, m64, m32,
                                                    mnorm);
 }
 
@@ -1192,12 +1194,14 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
 #undef WK_FUSED
       return after_launch(ctx);
     } else if (DF <= 8192) {
-      // warps per row: the fewest that leave a lane at most kRowMaxVpl 16-byte column groups
+      // warps per row: the fewest that leave a lane at most the mode's number of 16-byte column groups
       const int vecs = DF / 8;
+      const int nw = per_head ? kRowWarpsHead : kRowWarpsWhole;
+      const int max_vpl = per_head ? kRowMaxVplHead : kRowMaxVplWhole;
       int wpr = 1;
-      while (wpr < kRowWarps && (vecs + 32 * wpr - 1) / (32 * wpr) > kRowMaxVpl) wpr <<= 1;
+      while (wpr < nw && (vecs + 32 * wpr - 1) / (32 * wpr) > max_vpl) wpr <<= 1;
       const int vpl = (vecs + 32 * wpr - 1) / (32 * wpr);
-      const int n_sets = kRowWarps / wpr;
+      const int n_sets = nw / wpr;
       const int hs = per_head ? H : 1;
       const size_t smem_r = static_cast<size_t>(n_sets) * DF * sizeof(double);
       // rows per CTA: an even share of all chunks' anchor rows, and never so few that a chunk is cut into more slices
@@ -1207,14 +1211,22 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       const int64_t r_min = (T + max_parts - 2) / (max_parts - 1);
       if (R < r_min) R = r_min;
       const dim3 grid(static_cast<unsigned>((total + R - 1) / R));
-#define WK_ROWS(V) launch_rows<V>(grid, smem_r, s, K, stride, chunks, T, DF, hs, wpr, static_cast<int>(R), partial, max_parts, tickets, m64, m32, mnorm)
-      switch (vpl) {
-        case 1: WK_ROWS(1); break;
-        case 2: WK_ROWS(2); break;
-        case 3: WK_ROWS(3); break;
-        case 4: WK_ROWS(4); break;
-        case 5: WK_ROWS(5); break;
-        default: WK_ROWS(6); break;
+#define WK_ROWS(V, W) launch_rows<V, W>(grid, smem_r, s, K, stride, chunks, T, DF, hs, wpr, static_cast<int>(R), partial, max_parts, tickets, m64, m32, mnorm)
+      if (per_head) {
+        switch (vpl) {
+          case 1: WK_ROWS(1, kRowWarpsHead); break;
+          case 2: WK_ROWS(2, kRowWarpsHead); break;
+          default: WK_ROWS(3, kRowWarpsHead); break;
+        }
+      } else {
+        switch (vpl) {
+          case 1: WK_ROWS(1, kRowWarpsWhole); break;
+          case 2: WK_ROWS(2, kRowWarpsWhole); break;
+          case 3: WK_ROWS(3, kRowWarpsWhole); break;
+          case 4: WK_ROWS(4, kRowWarpsWhole); break;
+          case 5: WK_ROWS(5, kRowWarpsWhole); break;
+          default: WK_ROWS(6, kRowWarpsWhole); break;
+        }
       }
 #undef WK_ROWS
     } else {
