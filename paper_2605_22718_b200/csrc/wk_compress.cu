@@ -30,7 +30,6 @@ namespace {
 
 constexpr int kMaxNormParts = 32;     // pitch of the per-problem |m|^2 record in scratch (one share is used)
 constexpr int kScoreThreads = 256;
-constexpr int kScoreRowsPerCta = 32;   // head_score's block of rows; score_select / compress_fused get theirs at launch
 
 __device__ __forceinline__ double bf16_to_f64(uint32_t bits16) {
   return static_cast<double>(__uint_as_float(bits16 << 16));
@@ -1062,38 +1061,64 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
   for (int i = tid; i < (D >> 2); i += kScoreThreads) m[i] = __ldcg(msrc + i);
   __syncthreads();
   const int vecs = D >> 3;
-  const int j0 = blockIdx.x * kScoreRowsPerCta;
-  const int j1 = min(NA, j0 + kScoreRowsPerCta);
+  const int rows = (NA + gridDim.x - 1) / gridDim.x;   // the chunk's non-anchor rows in gridDim.x equal blocks
+  const int j0 = min(NA, static_cast<int>(blockIdx.x) * rows);
+  const int j1 = min(NA, j0 + rows);
   const __nv_bfloat16* Kb = K + static_cast<int64_t>(chunk) * stride + static_cast<int64_t>(T) * D;
   constexpr int W = kScoreThreads / 32;
-  for (int j = j0 + warp; j < j1; j += W) {
-    const uint4* row = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
+  // two rows per warp at a time, so that twice as many 16-byte loads are in flight
+  for (int j = j0 + warp; j < j1; j += 2 * W) {
+    const int jb = j + W;
+    const bool has_b = jb < j1;
+    const uint4* row_a = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(j) * D);
+    const uint4* row_b = reinterpret_cast<const uint4*>(Kb + static_cast<int64_t>(has_b ? jb : j) * D);
     for (int v0 = lane; v0 - lane < vecs; v0 += 128) {
-      uint4 q[4];
+      uint4 qa[4], qb[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) q[u] = v0 + 32 * u < vecs ? __ldg(row + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+      for (int u = 0; u < 4; ++u) {
+        const bool in = v0 + 32 * u < vecs;
+        qa[u] = in ? __ldg(row_a + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+        qb[u] = in ? __ldg(row_b + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
+      }
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + 32 * u;
-        float dot = 0.f, n2 = 0.f;
+        float dot_a = 0.f, n2_a = 0.f, dot_b = 0.f, n2_b = 0.f;
         if (v < vecs) {
+          // packed fp32 pairs, as in score_role: the low and the high halves of the words keep separate sums of four
+          // terms each, added once at the end (no deeper than the single chain of eight the error band was derived for)
           const float4 ma = m[2 * v], mb = m[2 * v + 1];
-          const float mm[8] = {ma.x, ma.y, ma.z, ma.w, mb.x, mb.y, mb.z, mb.w};
-          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+          const uint64_t mm[4] = {ptx::pack_f32x2(ma.x, ma.y), ptx::pack_f32x2(ma.z, ma.w), ptx::pack_f32x2(mb.x, mb.y),
+                                  ptx::pack_f32x2(mb.z, mb.w)};
+          const uint32_t wa[4] = {qa[u].x, qa[u].y, qa[u].z, qa[u].w}, wb[4] = {qb[u].x, qb[u].y, qb[u].z, qb[u].w};
+          uint64_t d2a = 0, s2a = 0, d2b = 0, s2b = 0;
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            float x;
-            x = bf16lo(w[e]); dot = fmaf(x, mm[2 * e], dot); n2 = fmaf(x, x, n2);
-            x = bf16hi(w[e]); dot = fmaf(x, mm[2 * e + 1], dot); n2 = fmaf(x, x, n2);
+            const uint64_t xa = ptx::pack_f32x2(bf16lo(wa[e]), bf16hi(wa[e]));
+            const uint64_t xb = ptx::pack_f32x2(bf16lo(wb[e]), bf16hi(wb[e]));
+            d2a = ptx::fma_f32x2(xa, mm[e], d2a);
+            s2a = ptx::fma_f32x2(xa, xa, s2a);
+            d2b = ptx::fma_f32x2(xb, mm[e], d2b);
+            s2b = ptx::fma_f32x2(xb, xb, s2b);
           }
+          float lo_, hi_;
+          ptx::unpack_f32x2(d2a, lo_, hi_); dot_a = lo_ + hi_;
+          ptx::unpack_f32x2(s2a, lo_, hi_); n2_a = lo_ + hi_;
+          ptx::unpack_f32x2(d2b, lo_, hi_); dot_b = lo_ + hi_;
+          ptx::unpack_f32x2(s2b, lo_, hi_); n2_b = lo_ + hi_;
         }
-        dot = half_warp_sum(dot);
-        n2 = half_warp_sum(n2);
+        dot_a = half_warp_sum(dot_a);
+        n2_a = half_warp_sum(n2_a);
+        dot_b = half_warp_sum(dot_b);
+        n2_b = half_warp_sum(n2_b);
         const int head = v >> 4;
-        if ((lane & 15) == 0 && head < H) {
+        // lanes 0 / 16 write row j's score of their head, lanes 1 / 17 row jb's
+        const int sel = lane & 15;
+        if (sel < 2 && head < H && (sel == 0 || has_b)) {
+          const float dot = sel ? dot_b : dot_a, n2 = sel ? n2_b : n2_a;
           const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
           if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
-          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + j;
+          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + (sel ? jb : j);
           s32[at] = sc;
           if (scores_out) scores_out[at] = sc;
         }
@@ -1240,7 +1265,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
                                                                 mnorm);
     }
     if ((st = after_launch(ctx)) != WK_OK) return st;
-    // score_select's blocks of rows: whole rounds of its 8 warps x 2 rows, and as few full waves of CTAs (four resident
+    // blocks of rows of score_select / head_score: whole rounds of its 8 warps x 2 rows, and as few full waves of CTAs (four resident
     // per SM) as blocks of at most 128 rows allow -- a last wave that is nearly empty costs as much as a full one
     int srows = 128;
     for (int waves = 1; waves <= 64; ++waves) {
@@ -1249,7 +1274,7 @@ wk_status launch_compress(wk_ctx* ctx, const __nv_bfloat16* K, int64_t stride, i
       const int r16 = static_cast<int>((per + 15) / 16 * 16);
       if (r16 <= 128) { srows = r16 < 16 ? 16 : r16; break; }
     }
-    const int nblk = per_head ? (NA + kScoreRowsPerCta - 1) / kScoreRowsPerCta : (NA + srows - 1) / srows;
+    const int nblk = (NA + srows - 1) / srows;
     if (per_head) {
       if (smem_m > 48 * 1024)
         WK_CUDA_TRY(ctx, cudaFuncSetAttribute(head_score, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem_m)));
