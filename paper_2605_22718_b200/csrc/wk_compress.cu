@@ -1080,6 +1080,8 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
         qa[u] = in ? __ldg(row_a + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
         qb[u] = in ? __ldg(row_b + v0 + 32 * u) : make_uint4(0, 0, 0, 0);
       }
+      // 16 partial sums per lane: for each of the four column groups u the pair (dot, |k|^2) of row j and of row jb
+      float val[16];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int v = v0 + 32 * u;
@@ -1107,21 +1109,37 @@ head_score(const __nv_bfloat16* __restrict__ K, int64_t stride, int T, int NA, i
           ptx::unpack_f32x2(d2b, lo_, hi_); dot_b = lo_ + hi_;
           ptx::unpack_f32x2(s2b, lo_, hi_); n2_b = lo_ + hi_;
         }
-        dot_a = half_warp_sum(dot_a);
-        n2_a = half_warp_sum(n2_a);
-        dot_b = half_warp_sum(dot_b);
-        n2_b = half_warp_sum(n2_b);
-        const int head = v >> 4;
-        // lanes 0 / 16 write row j's score of their head, lanes 1 / 17 row jb's
-        const int sel = lane & 15;
-        if (sel < 2 && head < H && (sel == 0 || has_b)) {
-          const float dot = sel ? dot_b : dot_a, n2 = sel ? n2_b : n2_a;
-          const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
-          if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
-          const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + (sel ? jb : j);
-          s32[at] = sc;
-          if (scores_out) scores_out[at] = sc;
+        val[4 * u + 0] = dot_a;
+        val[4 * u + 1] = n2_a;
+        val[4 * u + 2] = dot_b;
+        val[4 * u + 3] = n2_b;
+      }
+      // Sum over the 16 lanes that hold a head's 128 columns, all 16 sums at once: at every step a lane keeps the half of
+      // its sums that its lane bit selects and hands the other half to its partner (8 + 4 + 2 + 1 shuffles instead of
+      // 16 x 4); lane l of the half-warp ends with sum number l, added in the same butterfly order as half_warp_sum.
+#pragma unroll
+      for (int step = 0; step < 4; ++step) {
+        const int o = 8 >> step, n_keep_vals = 8 >> step;
+        const bool upper = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < n_keep_vals; ++i) {
+          const float keep = upper ? val[i + n_keep_vals] : val[i];
+          const float send = upper ? val[i] : val[i + n_keep_vals];
+          val[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
         }
+      }
+      // sum number l = 4 u + k: k = 0 / 2 are the dots of rows j / jb, their squared norms sit one lane up
+      const float n2 = __shfl_down_sync(0xffffffffu, val[0], 1);
+      const int l16 = lane & 15, u_of = l16 >> 2, k_of = l16 & 3;
+      const int v_of = v0 - lane + 32 * u_of + (lane & 16);   // a column group of this lane's half-warp and group u_of
+      const int head = v_of >> 4;
+      if ((k_of & 1) == 0 && v_of < vecs && head < H && (k_of == 0 || has_b)) {
+        const float dot = val[0];
+        const float sc = n2 == 0.f ? 0.f : __fdiv_rn(dot, __fsqrt_rn(n2));   // a NaN norm stays NaN and is reported
+        if (!isfinite(sc)) atomicOr(status, WK_DEV_NONFINITE);
+        const int64_t at = (static_cast<int64_t>(chunk) * H + head) * NA + (k_of ? jb : j);
+        s32[at] = sc;
+        if (scores_out) scores_out[at] = sc;
       }
     }
   }
