@@ -26,13 +26,27 @@ append_rows(const __nv_bfloat16* __restrict__ Ksrc, const __nv_bfloat16* __restr
   const int r0 = blockIdx.x * rows_per_cta, r1 = min(C, r0 + rows_per_cta);
   for (int r = r0 + warp; r < r1; r += kAppendThreads / 32) {
     uint4* d = reinterpret_cast<uint4*>(dst + static_cast<int64_t>(r) * D);
-    for (int v = lane; v < vecs; v += 32) {
-      const int j = idx[(v / vecs_per_list) * C + r];
-      if (j < 0 || j >= FT) {                     // never dereference a bad index
-        atomicOr(status, WK_DEV_BAD_SLOT);
-        continue;
+    // four 16-byte loads of the row in flight per lane before the first store
+    for (int v0 = lane; v0 < vecs; v0 += 128) {
+      uint4 q[4];
+      bool ok[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int v = v0 + 32 * u;
+        ok[u] = v < vecs;
+        if (ok[u]) {
+          const int j = idx[(v / vecs_per_list) * C + r];
+          if (j < 0 || j >= FT) {                   // never dereference a bad index
+            atomicOr(status, WK_DEV_BAD_SLOT);
+            ok[u] = false;
+          } else {
+            q[u] = __ldg(reinterpret_cast<const uint4*>(src + static_cast<int64_t>(j) * D) + v);
+          }
+        }
       }
-      d[v] = __ldg(reinterpret_cast<const uint4*>(src + static_cast<int64_t>(j) * D) + v);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (ok[u]) d[v0 + 32 * u] = q[u];
     }
   }
 }
