@@ -41,6 +41,7 @@ def test_device_generators_match_numpy():
     (200, 16, 100, 3, 0.1),       # 2,048 columns: two warps share a row of the anchor pass
     (96, 13, 48, 2, 0.1),         # 1,664 columns: two warps per row, some lanes without a column group
     (45, 20, 30, 5, 0.1),         # wide rows, several short chunks
+    (4, 2, 4, 400, 0.1),          # hundreds of tiny chunks: a CTA's run of anchor rows crosses three or four of them
 ])
 def test_compress_matches_oracle(T, H, n_keep, batch, sigma):
     D = H * 128
